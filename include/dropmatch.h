@@ -1,0 +1,153 @@
+/*
+ * dropmatch.h -- C ABI of the B200 (sm_100a) DropMatch verification library.
+ *
+ * DropMatch (arXiv 2603.03333) verifies draft tokens of speculative decoding by
+ * Monte-Carlo dropout on the LM head only.  For every draft position t the target
+ * model's final hidden state h_t[d] is copied K times, each copy multiplied by an
+ * independent Bernoulli(1-p) keep mask and rescaled by 1/(1-p) (Eq. 1, Eq. 2);
+ * each copy is projected through the shared head W[V,d] (Eq. 3) and decoded to its
+ * argmax token (Sec. 3.2).  The K tokens of a position form an empirical token
+ * distribution; a draft token is accepted when it is one of them (naive
+ * token-matching criterion, Sec. 3.2) or when it is their most frequent token
+ * (majority criterion, Eq. 6).  Positions are accepted left to right and the first
+ * rejection rejects everything after it (Sec. 2, lossless-decoding paragraph);
+ * for draft trees (Sec. 4.4) the result is the longest accepted root-to-leaf path.
+ *
+ * Conventions that hold for every entry point
+ *   - Unless a parameter says "host", every tensor pointer is a DEVICE pointer on
+ *     the context's device, owned by the caller, dense row-major, and must stay
+ *     valid until the work queued on `stream` has finished.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Device-pointer entry points only enqueue work: they never
+ *     synchronise, never allocate and never free.
+ *   - The library allocates device memory only in dm_create / dm_set_head (its
+ *     workspace) and frees it in dm_set_head / dm_destroy.
+ *   - Every function returns DM_OK or a negative status; nothing throws, aborts
+ *     or prints.  A CUDA error raised by earlier asynchronous work is reported by
+ *     the next call as DM_ECUDA.  A kernel that gives up on an internal wait sets
+ *     the context's device error word, which dm_device_error() reads.
+ *   - Masks: element j of path i at position t of sequence s is dropped iff word
+ *     (j mod 4) of Philox4x32-10(counter = (j/4, i, t, s mod 2^32),
+ *     key = (seed low 32 bits, seed high 32 bits)) is < floor(p * 2^32).
+ *     Results depend on (seed, s, t, i, j) only, never on batching or launch shape.
+ *   - Row order: path i of hidden row q (q = b*T + t) is "row" q*K + i.
+ *   - A context is not thread-safe; use one per host thread or lock around it.
+ */
+#ifndef DROPMATCH_H_
+#define DROPMATCH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dm_ctx dm_ctx; /* opaque: device id, head description, workspace, TMA descriptors */
+
+enum {
+    DM_OK = 0,
+    DM_EINVAL = -1,       /* bad argument (null pointer, size < 1, p outside [0,1), bad enum)   */
+    DM_EUNSUPPORTED = -2, /* shape the kernels cannot handle (see dm_set_head)                  */
+    DM_ECUDA = -3,        /* a CUDA runtime or driver call failed                               */
+    DM_EWORKSPACE = -4,   /* call needs more rows than dm_set_head reserved                     */
+    DM_EDEVICE = -5,      /* device is not compute capability 10.x                              */
+    DM_ENOHEAD = -6       /* dm_set_head has not been called                                    */
+};
+enum { DM_F32 = 0, DM_BF16 = 1 };             /* storage type of W and H (accumulation is fp32) */
+enum { DM_RULE_NAIVE = 0, DM_RULE_MAJORITY = 1 };
+enum { DM_IMPL_AUTO = 0, DM_IMPL_SIMT = 1, DM_IMPL_TCGEN05 = 2 };
+
+/* Create a context on CUDA device `device` (must be sm_100).  *out is set on success. */
+int dm_create(dm_ctx** out, int device);
+/* Free the context and its workspace.  Synchronises the device first.  NULL is allowed. */
+int dm_destroy(dm_ctx* ctx);
+
+/* Describe the LM head (Eq. 3): W is a device pointer to V*d elements, row-major [V,d],
+ * 16-byte aligned, caller-owned; it is read, never written, by every verify call until the
+ * next dm_set_head.  Reserves workspace for calls of up to `max_rows` rows (rows = B*T*K, or
+ * B*N_h*K for trees) and `max_hidden_rows` = rows/K hidden rows (used only by the *_host entry
+ * point's staging buffers).  Requirements: V >= 1; d >= 4 and d % 4 == 0 (fp32) or d % 8 == 0
+ * (bf16); else DM_EUNSUPPORTED.  bf16 heads with d % 64 == 0 run on the tcgen05 tensor-core
+ * kernel, everything else on the CUDA-core kernel.  Synchronises the device (re-allocation). */
+int dm_set_head(dm_ctx* ctx, const void* W, int V, int d, int dtype, int max_rows, int max_hidden_rows);
+
+/* Force a kernel family (DM_IMPL_*) for later calls; DM_IMPL_AUTO restores the default choice.
+ * DM_IMPL_TCGEN05 on a head it cannot handle makes verify calls return DM_EUNSUPPORTED. */
+int dm_set_impl(dm_ctx* ctx, int impl);
+
+/* Verify one chain of T draft tokens (sequence id 0): Eq. 1-3, per-path argmax, token counts,
+ * acceptance scan.
+ *   H[T,d]           hidden state whose head output predicts draft[t] (storage type of the head)
+ *   draft[T]         draft token ids (ids outside [0,V) simply never match)
+ *   K                paths per position, 1 <= K <= 1024;  p in [0,1): drop probability;  seed: Philox key
+ *   rule             DM_RULE_NAIVE (Sec. 3.2 token matching) or DM_RULE_MAJORITY (Eq. 6)
+ *   out_tokens[T,K]  argmax token of every path (ties: smallest id)
+ *   out_counts[T,K]  out_counts[t,i] = number of paths i' with out_tokens[t,i'] == out_tokens[t,i]
+ *   out_accept_len[1] number of leading accepted draft tokens, in [0,T] */
+int dropmatch_verify(dm_ctx* ctx, const void* H, const int32_t* draft, int T, int K, float p,
+                     uint64_t seed, int rule, int32_t* out_tokens, int32_t* out_counts,
+                     int32_t* out_accept_len, void* stream);
+
+/* B independent chains in one pass over W; sequence b has id seq_base + b.
+ *   H[B,T,d], draft[B,T] -> out_tokens[B,T,K], out_counts[B,T,K], out_accept_len[B];
+ *   out_draft_hits[B,T] (may be NULL) = number of paths whose token equals draft[b,t].
+ * Equals B calls of dropmatch_verify with the matching sequence ids, bit for bit. */
+int dropmatch_verify_batched(dm_ctx* ctx, const void* H, const int32_t* draft, int B, int T, int K,
+                             float p, uint64_t seed, uint64_t seq_base, int rule,
+                             int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
+                             int32_t* out_accept_len, void* stream);
+
+/* Same as dropmatch_verify_batched, but H, draft and all outputs are HOST pointers (pinned or
+ * pageable).  Copies the inputs to the device, runs the call, copies the outputs back and waits
+ * for `stream`.  Needs B*T <= max_hidden_rows of dm_set_head.  out_draft_hits may be NULL. */
+int dropmatch_verify_batched_host(dm_ctx* ctx, const void* H_host, const int32_t* draft_host, int B,
+                                  int T, int K, float p, uint64_t seed, uint64_t seq_base, int rule,
+                                  int32_t* out_tokens_host, int32_t* out_counts_host,
+                                  int32_t* out_draft_hits_host, int32_t* out_accept_len_host,
+                                  void* stream);
+
+/* Draft trees (Sec. 4.4).  Per sequence: N_h hidden rows H[b,q,:] and N nodes in topological
+ * order.  Node n has a token, a parent node (node_parent[n] < n; -1 = child of the committed
+ * prefix) and node_hrow[n] in [0,N_h): the hidden row whose head output predicts it (children
+ * of one parent share one row).  Paths of hidden row q use position index t = q in the mask key.
+ *   node_ok[n] = (parent is the prefix or node_ok[parent]) and token[n] passes `rule` against the
+ *                K tokens of row node_hrow[n];
+ *   out_accept_len[b] = depth of the deepest ok node (0 if none);
+ *   out_best_node[b]  = smallest-index ok node of that depth (-1 if none).
+ *   out_tokens[B,N_h,K], out_counts[B,N_h,K]; out_node_ok[B,N] may be NULL.
+ * Node arrays are not validated on the device beyond clamping out-of-range indices to "rejected". */
+int dropmatch_verify_tree(dm_ctx* ctx, const void* H, const int32_t* node_token,
+                          const int32_t* node_parent, const int32_t* node_hrow, int B, int N_h, int N,
+                          int K, float p, uint64_t seed, uint64_t seq_base, int rule,
+                          int32_t* out_tokens, int32_t* out_counts, int32_t* out_node_ok,
+                          int32_t* out_best_node, int32_t* out_accept_len, void* stream);
+
+/* Debug: full logits (Eq. 3 with Eq. 2's scale) of selected paths, computed by the same kernel
+ * family a verify call would use.  H[B,T,d]; row_sel[n_sel,3] holds (b, t, i) triples with
+ * 0 <= b < B, 0 <= t < T, i >= 0 (checked on the device: a bad triple yields a row of NaN);
+ * sequence b has id seq_base + b.  out_logits[n_sel,V] fp32.  1 <= n_sel <= max_rows. */
+int dm_debug_logits(dm_ctx* ctx, const void* H, int B, int T, const int32_t* row_sel, int n_sel,
+                    float p, uint64_t seed, uint64_t seq_base, float* out_logits, void* stream);
+
+/* Debug: the keep masks of Eq. 1, bit-packed.  out_bits[B,T,K,ceil(d/32)]: bit (j mod 32) of
+ * word j/32 is 1 iff element j is kept.  Needs no head. */
+int dm_debug_masks(dm_ctx* ctx, int B, int T, int K, int d, float p, uint64_t seed,
+                   uint64_t seq_base, uint32_t* out_bits, void* stream);
+
+/* Reads and clears the context's device error word (0 = none); synchronises `stream` first.
+ * Non-zero means a kernel abandoned an internal wait and the outputs of that call are invalid. */
+int dm_device_error(dm_ctx* ctx, void* stream, uint32_t* out_code);
+
+/* Bytes of device workspace the context holds; which kernel family the last verify call used
+ * (DM_IMPL_SIMT or DM_IMPL_TCGEN05, 0 before any call); kernels launched by the last call. */
+size_t dm_workspace_bytes(const dm_ctx* ctx);
+int dm_last_impl(const dm_ctx* ctx);
+int dm_last_launches(const dm_ctx* ctx);
+
+const char* dm_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DROPMATCH_H_ */

@@ -1,0 +1,218 @@
+"""Thin ctypes binding of libdropmatch's C ABI (include/dropmatch.h).
+
+Argument marshalling only: torch tensors give device pointers and the current stream; every
+step of the verification path runs inside the library's CUDA kernels.  There is no CPU
+fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+OK, EINVAL, EUNSUPPORTED, ECUDA, EWORKSPACE, EDEVICE, ENOHEAD = 0, -1, -2, -3, -4, -5, -6
+F32, BF16 = 0, 1
+RULE_NAIVE, RULE_MAJORITY = 0, 1
+IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+
+_LIB_PATH = Path(__file__).resolve().parent / "libdropmatch.so"
+_lib = None
+
+_vp, _ci, _cf, _u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_uint64
+
+# name -> (restype, argtypes); mirrors include/dropmatch.h declaration by declaration
+SIGNATURES = {
+    "dm_create": (_ci, [ctypes.POINTER(_vp), _ci]),
+    "dm_destroy": (_ci, [_vp]),
+    "dm_set_head": (_ci, [_vp, _vp, _ci, _ci, _ci, _ci, _ci]),
+    "dm_set_impl": (_ci, [_vp, _ci]),
+    "dropmatch_verify": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _u64, _ci, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_batched": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_batched_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_tree": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
+                                    _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
+    "dm_debug_masks": (_ci, [_vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
+    "dm_device_error": (_ci, [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]),
+    "dm_workspace_bytes": (ctypes.c_size_t, [_vp]),
+    "dm_last_impl": (_ci, [_vp]),
+    "dm_last_launches": (_ci, [_vp]),
+    "dm_strerror": (ctypes.c_char_p, [_ci]),
+}
+
+
+class DropMatchError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libdropmatch.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -c 'import __graft_entry__ as g; g.build()'`")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().dm_strerror(status).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise DropMatchError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, what: str) -> torch.Tensor:
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{what} must be a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+class Context:
+    """One dm_ctx: a device, an LM head, and the library-owned workspace."""
+
+    def __init__(self, device: int = 0):
+        self._h = ctypes.c_void_p()
+        self.device = torch.device("cuda", device)
+        _check(lib().dm_create(ctypes.byref(self._h), device), "dm_create")
+        self._W = None
+        self.dtype = None
+
+    def close(self):
+        if self._h:
+            lib().dm_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _tdtype(self):
+        return torch.float32 if self.dtype == F32 else torch.bfloat16
+
+    # -- dm_set_head / dm_set_impl
+    def set_head(self, W: torch.Tensor, max_rows: int, max_hidden_rows: int | None = None):
+        if W.dtype not in (torch.float32, torch.bfloat16) or not W.is_cuda or not W.is_contiguous() or W.dim() != 2:
+            raise TypeError("W must be a contiguous 2-D CUDA tensor of float32 or bfloat16")
+        dtype = F32 if W.dtype == torch.float32 else BF16
+        V, d = W.shape
+        _check(lib().dm_set_head(self._h, _ptr(W), V, d, dtype, max_rows, max_hidden_rows or max_rows), "dm_set_head")
+        self._W, self.dtype, self.V, self.d = W, dtype, V, d   # keep W alive
+
+    def set_impl(self, impl: int):
+        _check(lib().dm_set_impl(self._h, impl), "dm_set_impl")
+
+    # -- dropmatch_verify
+    def verify(self, H, draft, K, p, seed, rule=RULE_NAIVE):
+        T = H.shape[0]
+        _dev(H, self._tdtype(), "H"); _dev(draft, torch.int32, "draft")
+        tokens = torch.empty((T, K), dtype=torch.int32, device=self.device)
+        counts = torch.empty_like(tokens)
+        alen = torch.empty((1,), dtype=torch.int32, device=self.device)
+        _check(lib().dropmatch_verify(self._h, _ptr(H), _ptr(draft), T, K, p, seed, rule, _ptr(tokens),
+                                      _ptr(counts), _ptr(alen), _stream(self.device)), "dropmatch_verify")
+        return dict(tokens=tokens, counts=counts, accept_len=alen)
+
+    # -- dropmatch_verify_batched
+    def verify_batched(self, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE, out=None):
+        B, T, _ = H.shape
+        _dev(H, self._tdtype(), "H"); _dev(draft, torch.int32, "draft")
+        if out is None:
+            out = self.alloc_outputs(B, T, K)
+        _check(lib().dropmatch_verify_batched(self._h, _ptr(H), _ptr(draft), B, T, K, p, seed, seq_base, rule,
+                                              _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["hits"]),
+                                              _ptr(out["accept_len"]), _stream(self.device)),
+               "dropmatch_verify_batched")
+        return out
+
+    def alloc_outputs(self, B, T, K):
+        i32 = dict(dtype=torch.int32, device=self.device)
+        return dict(tokens=torch.empty((B, T, K), **i32), counts=torch.empty((B, T, K), **i32),
+                    hits=torch.empty((B, T), **i32), accept_len=torch.empty((B,), **i32))
+
+    # -- dropmatch_verify_batched_host
+    def verify_batched_host(self, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE, out=None):
+        """H, draft and outputs are CPU tensors (pinned for speed); returns after the results are on the host."""
+        B, T, _ = H.shape
+        if H.is_cuda or draft.is_cuda or not H.is_contiguous() or not draft.is_contiguous():
+            raise TypeError("host entry point takes contiguous CPU tensors")
+        if H.dtype != self._tdtype() or draft.dtype != torch.int32:
+            raise TypeError("H must have the head's dtype and draft must be int32")
+        if out is None:
+            out = self.alloc_host_outputs(B, T, K)
+        _check(lib().dropmatch_verify_batched_host(self._h, _ptr(H), _ptr(draft), B, T, K, p, seed, seq_base, rule,
+                                                   _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["hits"]),
+                                                   _ptr(out["accept_len"]), _stream(self.device)),
+               "dropmatch_verify_batched_host")
+        return out
+
+    @staticmethod
+    def alloc_host_outputs(B, T, K, pin=True):
+        mk = lambda *s: torch.empty(s, dtype=torch.int32, pin_memory=pin)
+        return dict(tokens=mk(B, T, K), counts=mk(B, T, K), hits=mk(B, T), accept_len=mk(B))
+
+    # -- dropmatch_verify_tree
+    def verify_tree(self, H, node_token, node_parent, node_hrow, K, p, seed, seq_base=0, rule=RULE_NAIVE):
+        B, N_h, _ = H.shape
+        N = node_token.shape[1]
+        _dev(H, self._tdtype(), "H")
+        for name, t in (("node_token", node_token), ("node_parent", node_parent), ("node_hrow", node_hrow)):
+            _dev(t, torch.int32, name)
+        i32 = dict(dtype=torch.int32, device=self.device)
+        out = dict(tokens=torch.empty((B, N_h, K), **i32), counts=torch.empty((B, N_h, K), **i32),
+                   node_ok=torch.empty((B, N), **i32), best_node=torch.empty((B,), **i32),
+                   accept_len=torch.empty((B,), **i32))
+        _check(lib().dropmatch_verify_tree(self._h, _ptr(H), _ptr(node_token), _ptr(node_parent), _ptr(node_hrow),
+                                           B, N_h, N, K, p, seed, seq_base, rule, _ptr(out["tokens"]),
+                                           _ptr(out["counts"]), _ptr(out["node_ok"]), _ptr(out["best_node"]),
+                                           _ptr(out["accept_len"]), _stream(self.device)), "dropmatch_verify_tree")
+        return out
+
+    # -- debug
+    def debug_logits(self, H, row_sel, p, seed, seq_base=0):
+        B, T, _ = H.shape
+        _dev(H, self._tdtype(), "H"); _dev(row_sel, torch.int32, "row_sel")
+        n = row_sel.shape[0]
+        out = torch.empty((n, self.V), dtype=torch.float32, device=self.device)
+        _check(lib().dm_debug_logits(self._h, _ptr(H), B, T, _ptr(row_sel), n, p, seed, seq_base, _ptr(out),
+                                     _stream(self.device)), "dm_debug_logits")
+        return out
+
+    def debug_masks(self, B, T, K, d, p, seed, seq_base=0):
+        out = torch.empty((B, T, K, (d + 31) // 32), dtype=torch.int32, device=self.device)
+        _check(lib().dm_debug_masks(self._h, B, T, K, d, p, seed, seq_base, _ptr(out), _stream(self.device)),
+               "dm_debug_masks")
+        return out
+
+    def device_error(self) -> int:
+        code = ctypes.c_uint32()
+        _check(lib().dm_device_error(self._h, _stream(self.device), ctypes.byref(code)), "dm_device_error")
+        return code.value
+
+    def workspace_bytes(self) -> int:
+        return lib().dm_workspace_bytes(self._h)
+
+    def last_impl(self) -> int:
+        return lib().dm_last_impl(self._h)
+
+    def last_launches(self) -> int:
+        return lib().dm_last_launches(self._h)

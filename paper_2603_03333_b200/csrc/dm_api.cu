@@ -1,0 +1,350 @@
+// C ABI of libdropmatch: argument checks, workspace, kernel choice.  See include/dropmatch.h.
+#include <math.h>
+#include <new>
+
+#include "dm_internal.h"
+
+using namespace dm;
+
+struct dm_ctx {
+    int device = 0;
+    HeadDesc head{nullptr, 0, 0, 0};
+    bool has_head = false;
+    int max_rows = 0, max_hidden = 0;
+    int impl = DM_IMPL_AUTO;
+    int last_impl = 0, last_launches = 0;
+    // workspace (device)
+    unsigned long long* partials = nullptr;  // [kMaxSlices][max_rows]
+    uint32_t* err = nullptr;                 // device error word
+    unsigned char* stage_H = nullptr;        // [max_hidden][d] storage type
+    int32_t* stage_i32 = nullptr;            // draft | tokens | counts | hits | accept_len
+    size_t ws_bytes = 0;
+    FusedState* fused = nullptr;             // tensor maps etc. of the tcgen05 kernel
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        target = dev;
+    }
+    ~DeviceGuard() { if (prev >= 0 && prev != target) cudaSetDevice(prev); }
+    int target = -1;
+};
+
+void free_workspace(dm_ctx* c) {
+    cudaFree(c->partials); c->partials = nullptr;
+    cudaFree(c->stage_H); c->stage_H = nullptr;
+    cudaFree(c->stage_i32); c->stage_i32 = nullptr;
+    if (c->fused) { fused_destroy(c->fused); c->fused = nullptr; }
+    c->ws_bytes = 0;
+}
+
+bool make_mask_key(float p, uint64_t seed, MaskKey* mk) {
+    if (!(p >= 0.0f) || !(p < 1.0f)) return false;
+    double scaled = floor((double)p * 4294967296.0);
+    if (scaled > 4294967295.0) scaled = 4294967295.0;
+    mk->thr = (uint32_t)scaled;
+    mk->key0 = (uint32_t)seed;
+    mk->key1 = (uint32_t)(seed >> 32);
+    mk->scale = (float)(1.0 / (1.0 - (double)p));
+    return true;
+}
+
+// Which kernel family serves this head under the context's override?
+int pick_impl(const dm_ctx* c, int rows, int* impl) {
+    const bool tc_ok = fused_supported(c->head, rows);
+    if (c->impl == DM_IMPL_TCGEN05) {
+        if (!tc_ok) return DM_EUNSUPPORTED;
+        *impl = DM_IMPL_TCGEN05;
+    } else if (c->impl == DM_IMPL_SIMT) {
+        *impl = DM_IMPL_SIMT;
+    } else {
+        *impl = tc_ok ? DM_IMPL_TCGEN05 : DM_IMPL_SIMT;
+    }
+    return DM_OK;
+}
+
+// Masked head + per-slice argmax for `rows` rows, then merge/histogram/acceptance.
+int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const MaskKey& mk,
+               const FinalizeArgs& fa, cudaStream_t stream) {
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    if (rows > c->max_rows) return DM_EWORKSPACE;
+    if (finalize_smem_bytes(fa.T, fa.K, fa.N) > 200 * 1024) return DM_EUNSUPPORTED;
+    int impl;
+    int st = pick_impl(c, rows, &impl);
+    if (st != DM_OK) return st;
+    int n_slices = 0, launches = 0;
+    if (impl == DM_IMPL_TCGEN05)
+        st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
+                          nullptr, c->err, stream, &launches);
+    else {
+        st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, stream);
+        launches = 1;
+    }
+    if (st != DM_OK) return st;
+    st = launch_finalize(c->partials, n_slices, rows, fa, stream);
+    if (st != DM_OK) return st;
+    c->last_impl = impl;
+    c->last_launches = launches + 1;
+    return DM_OK;
+}
+
+int check_common(const dm_ctx* c, const void* H, int B, int T, int K) {
+    if (c == nullptr || H == nullptr) return DM_EINVAL;
+    if (!c->has_head) return DM_ENOHEAD;
+    if (B < 1 || T < 1 || K < 1 || K > kMaxK) return DM_EINVAL;
+    if ((long long)B * T * K > 0x3FFFFFFFll) return DM_EINVAL;
+    return DM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dm_create(dm_ctx** out, int device) {
+    if (out == nullptr) return DM_EINVAL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    if (device < 0 || device >= count) return DM_EINVAL;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return DM_ECUDA;
+    if (major != 10) return DM_EDEVICE;
+    DeviceGuard g(device);
+    if (!g.ok) return DM_ECUDA;
+    dm_ctx* c = new (std::nothrow) dm_ctx();
+    if (c == nullptr) return DM_ECUDA;
+    c->device = device;
+    if (cudaMalloc(&c->err, sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(c->err, 0, sizeof(uint32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(c->err);
+        delete c;
+        return DM_ECUDA;
+    }
+    *out = c;
+    return DM_OK;
+}
+
+int dm_destroy(dm_ctx* c) {
+    if (c == nullptr) return DM_OK;
+    DeviceGuard g(c->device);
+    cudaDeviceSynchronize();
+    free_workspace(c);
+    cudaFree(c->err);
+    cudaGetLastError();
+    delete c;
+    return DM_OK;
+}
+
+int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows, int max_hidden_rows) {
+    if (c == nullptr || W == nullptr) return DM_EINVAL;
+    if (dtype != DM_F32 && dtype != DM_BF16) return DM_EINVAL;
+    if (V < 1 || d < 1 || max_rows < 1 || max_hidden_rows < 1) return DM_EINVAL;
+    if (max_rows > (1 << 24) || max_hidden_rows > max_rows) return DM_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(W) & 15u) != 0) return DM_EINVAL;
+    const int vec = dtype == DM_F32 ? 4 : 8;
+    if (d < 4 || d % vec != 0) return DM_EUNSUPPORTED;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    free_workspace(c);
+    c->has_head = false;
+    const size_t elem = dtype == DM_F32 ? 4 : 2;
+    const size_t n_part = (size_t)kMaxSlices * max_rows * sizeof(unsigned long long);
+    const size_t n_H = (size_t)max_hidden_rows * d * elem;
+    const size_t n_i32 = ((size_t)3 * max_hidden_rows + 2 * (size_t)max_rows) * sizeof(int32_t);
+    if (cudaMalloc(&c->partials, n_part) != cudaSuccess || cudaMalloc(&c->stage_H, n_H) != cudaSuccess ||
+        cudaMalloc(&c->stage_i32, n_i32) != cudaSuccess) {
+        cudaGetLastError();
+        free_workspace(c);
+        return DM_ECUDA;
+    }
+    c->ws_bytes = n_part + n_H + n_i32;
+    c->head = HeadDesc{W, V, d, dtype};
+    c->max_rows = max_rows;
+    c->max_hidden = max_hidden_rows;
+    size_t fused_bytes = 0;
+    int st = fused_create(&c->fused, c->head, max_rows, max_hidden_rows, &fused_bytes);
+    if (st != DM_OK) { free_workspace(c); return st; }
+    c->ws_bytes += fused_bytes;
+    c->has_head = true;
+    return DM_OK;
+}
+
+int dm_set_impl(dm_ctx* c, int impl) {
+    if (c == nullptr || impl < DM_IMPL_AUTO || impl > DM_IMPL_TCGEN05) return DM_EINVAL;
+    c->impl = impl;
+    return DM_OK;
+}
+
+int dropmatch_verify_batched(dm_ctx* c, const void* H, const int32_t* draft, int B, int T, int K,
+                             float p, uint64_t seed, uint64_t seq_base, int rule, int32_t* out_tokens,
+                             int32_t* out_counts, int32_t* out_draft_hits, int32_t* out_accept_len,
+                             void* stream) {
+    int st = check_common(c, H, B, T, K);
+    if (st != DM_OK) return st;
+    if (draft == nullptr || out_tokens == nullptr || out_counts == nullptr || out_accept_len == nullptr)
+        return DM_EINVAL;
+    if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base};
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = T; fa.K = K; fa.rule = rule;
+    fa.draft = draft; fa.out_hits = out_draft_hits;
+    fa.N = 0;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    return run_verify(c, H, B * T * K, map, mk, fa, static_cast<cudaStream_t>(stream));
+}
+
+int dropmatch_verify(dm_ctx* c, const void* H, const int32_t* draft, int T, int K, float p,
+                     uint64_t seed, int rule, int32_t* out_tokens, int32_t* out_counts,
+                     int32_t* out_accept_len, void* stream) {
+    return dropmatch_verify_batched(c, H, draft, 1, T, K, p, seed, 0, rule, out_tokens, out_counts,
+                                    nullptr, out_accept_len, stream);
+}
+
+int dropmatch_verify_batched_host(dm_ctx* c, const void* H_host, const int32_t* draft_host, int B, int T,
+                                  int K, float p, uint64_t seed, uint64_t seq_base, int rule,
+                                  int32_t* out_tokens_host, int32_t* out_counts_host,
+                                  int32_t* out_draft_hits_host, int32_t* out_accept_len_host,
+                                  void* stream) {
+    int st = check_common(c, H_host, B, T, K);
+    if (st != DM_OK) return st;
+    if (draft_host == nullptr || out_tokens_host == nullptr || out_counts_host == nullptr ||
+        out_accept_len_host == nullptr)
+        return DM_EINVAL;
+    const long long hidden = (long long)B * T, rows = hidden * K;
+    if (hidden > c->max_hidden || rows > c->max_rows) return DM_EWORKSPACE;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t elem = c->head.dtype == DM_F32 ? 4 : 2;
+    int32_t* d_draft = c->stage_i32;
+    int32_t* d_hits = d_draft + c->max_hidden;
+    int32_t* d_len = d_hits + c->max_hidden;
+    int32_t* d_tok = d_len + c->max_hidden;
+    int32_t* d_cnt = d_tok + c->max_rows;
+    if (cudaMemcpyAsync(c->stage_H, H_host, (size_t)hidden * c->head.d * elem, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(d_draft, draft_host, (size_t)hidden * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return DM_ECUDA;
+    }
+    st = dropmatch_verify_batched(c, c->stage_H, d_draft, B, T, K, p, seed, seq_base, rule, d_tok, d_cnt,
+                                  d_hits, d_len, stream);
+    if (st != DM_OK) return st;
+    bool ok = cudaMemcpyAsync(out_tokens_host, d_tok, (size_t)rows * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+              cudaMemcpyAsync(out_counts_host, d_cnt, (size_t)rows * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+              cudaMemcpyAsync(out_accept_len_host, d_len, (size_t)B * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    if (ok && out_draft_hits_host)
+        ok = cudaMemcpyAsync(out_draft_hits_host, d_hits, (size_t)hidden * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    if (!ok || cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    return DM_OK;
+}
+
+int dropmatch_verify_tree(dm_ctx* c, const void* H, const int32_t* node_token, const int32_t* node_parent,
+                          const int32_t* node_hrow, int B, int N_h, int N, int K, float p, uint64_t seed,
+                          uint64_t seq_base, int rule, int32_t* out_tokens, int32_t* out_counts,
+                          int32_t* out_node_ok, int32_t* out_best_node, int32_t* out_accept_len,
+                          void* stream) {
+    int st = check_common(c, H, B, N_h, K);
+    if (st != DM_OK) return st;
+    if (N < 1 || N > (1 << 20)) return DM_EINVAL;
+    if (node_token == nullptr || node_parent == nullptr || node_hrow == nullptr || out_tokens == nullptr ||
+        out_counts == nullptr || out_best_node == nullptr || out_accept_len == nullptr)
+        return DM_EINVAL;
+    if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    RowMap map{nullptr, K, N_h, B, (uint32_t)seq_base};
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = N_h; fa.K = K; fa.rule = rule;
+    fa.N = N; fa.node_token = node_token; fa.node_parent = node_parent; fa.node_hrow = node_hrow;
+    fa.out_node_ok = out_node_ok; fa.out_best_node = out_best_node;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    return run_verify(c, H, B * N_h * K, map, mk, fa, static_cast<cudaStream_t>(stream));
+}
+
+int dm_debug_logits(dm_ctx* c, const void* H, int B, int T, const int32_t* row_sel, int n_sel, float p,
+                    uint64_t seed, uint64_t seq_base, float* out_logits, void* stream) {
+    if (c == nullptr || H == nullptr || row_sel == nullptr || out_logits == nullptr) return DM_EINVAL;
+    if (!c->has_head) return DM_ENOHEAD;
+    if (B < 1 || T < 1 || n_sel < 1) return DM_EINVAL;
+    if (n_sel > c->max_rows) return DM_EWORKSPACE;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    RowMap map{row_sel, 1, T, B, (uint32_t)seq_base};
+    int impl;
+    int st = pick_impl(c, n_sel, &impl);
+    if (st != DM_OK) return st;
+    int n_slices = 0, launches = 1;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (impl == DM_IMPL_TCGEN05)
+        st = fused_launch(c->fused, c->head, H, B * T, n_sel, map, mk, &n_slices, c->partials, out_logits,
+                          c->err, s, &launches);
+    else
+        st = launch_simt(c->head, H, n_sel, map, mk, &n_slices, c->partials, out_logits, c->err, s);
+    if (st != DM_OK) return st;
+    c->last_impl = impl;
+    c->last_launches = launches;
+    return DM_OK;
+}
+
+int dm_debug_masks(dm_ctx* c, int B, int T, int K, int d, float p, uint64_t seed, uint64_t seq_base,
+                   uint32_t* out_bits, void* stream) {
+    if (c == nullptr || out_bits == nullptr) return DM_EINVAL;
+    if (B < 1 || T < 1 || K < 1 || d < 1) return DM_EINVAL;
+    if ((long long)B * T * K > 0x3FFFFFFFll) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    return launch_debug_masks(B, T, K, d, mk, (uint32_t)seq_base, out_bits, static_cast<cudaStream_t>(stream));
+}
+
+int dm_device_error(dm_ctx* c, void* stream, uint32_t* out_code) {
+    if (c == nullptr || out_code == nullptr) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t code = 0;
+    if (cudaMemcpyAsync(&code, c->err, sizeof code, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemsetAsync(c->err, 0, sizeof code, s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return DM_ECUDA;
+    }
+    *out_code = code;
+    return DM_OK;
+}
+
+size_t dm_workspace_bytes(const dm_ctx* c) { return c ? c->ws_bytes : 0; }
+int dm_last_impl(const dm_ctx* c) { return c ? c->last_impl : 0; }
+int dm_last_launches(const dm_ctx* c) { return c ? c->last_launches : 0; }
+
+const char* dm_strerror(int status) {
+    switch (status) {
+        case DM_OK: return "ok";
+        case DM_EINVAL: return "invalid argument";
+        case DM_EUNSUPPORTED: return "unsupported shape";
+        case DM_ECUDA: return "CUDA error";
+        case DM_EWORKSPACE: return "call exceeds the rows reserved by dm_set_head";
+        case DM_EDEVICE: return "device is not compute capability 10.x";
+        case DM_ENOHEAD: return "dm_set_head has not been called";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,69 @@
+// Internal host-side declarations shared by the translation units of libdropmatch.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dropmatch.h"
+#include "dm_common.cuh"
+
+namespace dm {
+
+constexpr int kSimtMaxSlices = 296;   // vocabulary slices of the CUDA-core kernel
+constexpr int kMaxSlices = 296;       // rows of the partial-argmax workspace
+constexpr int kMaxK = 1024;
+
+struct HeadDesc {
+    const void* W;
+    int V, d, dtype;
+};
+
+// Per-call mask parameters (Eq. 1, Eq. 2).
+struct MaskKey {
+    uint32_t key0, key1;  // Philox key = seed
+    uint32_t thr;         // drop iff word < thr; thr = floor(p * 2^32)
+    float scale;          // 1 / (1 - p)
+};
+
+// Acceptance inputs/outputs handed to the finalize kernel.
+struct FinalizeArgs {
+    int B, T, K, rule;
+    // chain
+    const int32_t* draft;        // [B,T] or null (tree)
+    int32_t* out_hits;           // [B,T] or null
+    // tree
+    int N;                       // nodes per sequence (0 = chain)
+    const int32_t* node_token;   // [B,N]
+    const int32_t* node_parent;  // [B,N]
+    const int32_t* node_hrow;    // [B,N]
+    int32_t* out_node_ok;        // [B,N] or null
+    int32_t* out_best_node;      // [B]
+    // both
+    int32_t* out_tokens;         // [B,T,K]
+    int32_t* out_counts;         // [B,T,K]
+    int32_t* out_accept_len;     // [B]
+};
+
+int launch_simt(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
+                int* n_slices_out, unsigned long long* partials, float* dbg_logits, uint32_t* err,
+                cudaStream_t stream);
+
+// Merge the per-slice partial argmaxes into tokens, count them, run the acceptance scan.
+int launch_finalize(const unsigned long long* partials, int n_slices, int rows,
+                    const FinalizeArgs& a, cudaStream_t stream);
+size_t finalize_smem_bytes(int T, int K, int N);
+
+// tcgen05 tensor-core kernel (bf16 heads).  FusedState owns the TMA descriptors.
+struct FusedState;
+bool fused_supported(const HeadDesc& head, int rows);
+int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int max_hidden_rows, size_t* bytes);
+void fused_destroy(FusedState* fs);
+int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidden, int rows,
+                 const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
+                 float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out);
+
+int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo,
+                       uint32_t* out_bits, cudaStream_t stream);
+
+}  // namespace dm

@@ -1,0 +1,205 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle, element by
+element, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_03333_b200 as pk
+from paper_2603_03333_b200 import binding, workloads as wl
+from parity_util import NEAR_TIE, TOL_LOGIT_BF16, TOL_LOGIT_F32, check_chain, check_tree, to_np
+
+pytestmark = pytest.mark.gpu
+SEED = wl.MASK_SEED
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = pk.Context(0)
+    yield c
+    c.close()
+
+
+def _impls(ctx, cfg):
+    """Kernel families that can serve this head: always the CUDA-core one, plus tcgen05 for bf16, d % 64 == 0."""
+    out = [binding.IMPL_SIMT]
+    if cfg.dtype == wl.BF16 and cfg.d % 64 == 0:
+        out.append(binding.IMPL_TCGEN05)
+    return out
+
+
+def _run_chain(ctx, cfg, impl, rule=oracle.RULE_NAIVE, seq_base=0, work=None):
+    work = work or wl.make_workload(cfg, device=DEV)
+    ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+    ctx.set_impl(impl)
+    try:
+        got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=seq_base, rule=rule))
+        assert ctx.device_error() == 0
+        assert ctx.last_impl() == impl
+    finally:
+        ctx.set_impl(binding.IMPL_AUTO)
+    ref = oracle.verify_batched(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H),
+                                work.draft.cpu().numpy(), cfg.K, cfg.p, SEED, seq_base=seq_base, rule=rule)
+    n_diff = check_chain(got, ref, work.draft.cpu().numpy(), rule)
+    return got, ref, n_diff, work
+
+
+@pytest.mark.parametrize("shape", [(1, 4, 8, 256), (2, 3, 5, 200), (1, 1, 1, 4), (3, 2, 32, 4096), (1, 2, 3, 33)])
+@pytest.mark.parametrize("p", [0.0, 0.1, 0.5])
+def test_masks_bit_exact(ctx, shape, p):
+    B, T, K, d = shape
+    got = ctx.debug_masks(B, T, K, d, p, SEED, seq_base=7).cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, oracle.masks(B, T, K, d, p, SEED, 7))
+
+
+def test_toy_config_fp32(ctx):
+    cfg = wl.CONFIGS["toy"]
+    got, ref, n_diff, work = _run_chain(ctx, cfg, binding.IMPL_SIMT)
+    assert n_diff == 0   # fp32 head: no near-tie is expected to flip at this size
+    sel = torch.tensor([[0, t, i] for t in range(cfg.T) for i in (0, 3, 7)], dtype=torch.int32, device=DEV)
+    logits = ctx.debug_logits(work.H, sel, cfg.p, SEED).cpu().numpy()
+    Wn, Hn = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H)
+    for n, (b, t, i) in enumerate(sel.cpu().tolist()):
+        exp = oracle.logits_row(Wn, cfg.dtype, Hn[b, t], cfg.p, SEED, b, t, i)
+        assert np.abs(logits[n] - exp).max() < TOL_LOGIT_F32
+
+
+SMALL = [
+    # several vocabulary tiles with a ragged tail, several k-blocks, rows not a multiple of 16
+    wl.Config("bf16_a", d=512, V=3000, dtype=wl.BF16, B=2, T=3, K=8, p=0.1),
+    wl.Config("bf16_b", d=192, V=1111, dtype=wl.BF16, B=1, T=5, K=5, p=0.3),
+    wl.Config("bf16_c", d=1024, V=20000, dtype=wl.BF16, B=3, T=2, K=16, p=0.05),
+    wl.Config("bf16_k1", d=256, V=700, dtype=wl.BF16, B=1, T=1, K=1, p=0.2),
+    wl.Config("bf16_wide", d=64, V=130, dtype=wl.BF16, B=1, T=2, K=32, p=0.5),
+    wl.Config("bf16_odd_d", d=136, V=999, dtype=wl.BF16, B=1, T=3, K=4, p=0.1),      # CUDA-core only
+    wl.Config("f32_b", d=100, V=517, dtype=wl.F32, B=2, T=3, K=7, p=0.2, draft_mode="toy"),
+    wl.Config("bf16_rows200", d=256, V=2500, dtype=wl.BF16, B=5, T=5, K=8, p=0.1),
+    wl.Config("bf16_rows300", d=128, V=1500, dtype=wl.BF16, B=3, T=10, K=10, p=0.1),
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+@pytest.mark.parametrize("rule", [oracle.RULE_NAIVE, oracle.RULE_MAJORITY])
+def test_small_heads_all_impls(ctx, cfg, rule):
+    for impl in _impls(ctx, cfg):
+        got, ref, n_diff, work = _run_chain(ctx, cfg, impl, rule=rule, seq_base=3)
+        assert n_diff <= max(2, cfg.rows // 10)
+        sel_l = [[b, t, i] for b in range(cfg.B) for t in range(cfg.T) for i in (0, cfg.K - 1)][:12]
+        sel = torch.tensor(sel_l, dtype=torch.int32, device=DEV)
+        ctx.set_impl(impl)
+        logits = ctx.debug_logits(work.H, sel, cfg.p, SEED, seq_base=3).cpu().numpy()
+        ctx.set_impl(binding.IMPL_AUTO)
+        assert ctx.device_error() == 0
+        Wn, Hn = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H)
+        tol = TOL_LOGIT_F32 if cfg.dtype == wl.F32 else TOL_LOGIT_BF16
+        for n, (b, t, i) in enumerate(sel_l):
+            exp = oracle.logits_row(Wn, cfg.dtype, Hn[b, t], cfg.p, SEED, 3 + b, t, i)
+            assert np.abs(logits[n] - exp).max() < tol, (impl, b, t, i)
+
+
+def test_p_zero_is_greedy_verification(ctx):
+    cfg = wl.Config("p0", d=256, V=2000, dtype=wl.BF16, B=2, T=4, K=6, p=0.0)
+    for impl in _impls(ctx, cfg):
+        got, ref, n_diff, work = _run_chain(ctx, cfg, impl)
+        assert (got["tokens"] == got["tokens"][..., :1]).all()      # every path decodes the same token
+        assert (got["counts"] == cfg.K).all()
+
+
+def test_batched_equals_singles_and_chain_equals_path_tree(ctx):
+    cfg = wl.Config("bs", d=256, V=3000, dtype=wl.BF16, B=3, T=4, K=8, p=0.2)
+    work = wl.make_workload(cfg, device=DEV)
+    ctx.set_head(work.W, max_rows=cfg.rows)
+    for impl in _impls(ctx, cfg):
+        ctx.set_impl(impl)
+        full = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=10))
+        for b in range(cfg.B):
+            one = to_np(ctx.verify_batched(work.H[b:b + 1].contiguous(), work.draft[b:b + 1].contiguous(),
+                                           cfg.K, cfg.p, SEED, seq_base=10 + b))
+            for key in ("tokens", "counts", "hits", "accept_len"):
+                assert np.array_equal(one[key][0], full[key][b]), key
+        single = to_np(ctx.verify(work.H[0].contiguous(), work.draft[0].contiguous(), cfg.K, cfg.p, SEED))
+        ref0 = to_np(ctx.verify_batched(work.H[:1].contiguous(), work.draft[:1].contiguous(), cfg.K, cfg.p, SEED))
+        assert np.array_equal(single["tokens"], ref0["tokens"][0])
+        assert single["accept_len"][0] == ref0["accept_len"][0]
+        parent = torch.arange(-1, cfg.T - 1, dtype=torch.int32, device=DEV).repeat(cfg.B, 1).contiguous()
+        hrow = torch.arange(cfg.T, dtype=torch.int32, device=DEV).repeat(cfg.B, 1).contiguous()
+        tree = to_np(ctx.verify_tree(work.H, work.draft, parent, hrow, cfg.K, cfg.p, SEED, seq_base=10))
+        assert np.array_equal(tree["tokens"], full["tokens"])
+        assert np.array_equal(tree["accept_len"], full["accept_len"])
+        assert np.array_equal(tree["best_node"], full["accept_len"] - 1)
+        ctx.set_impl(binding.IMPL_AUTO)
+    assert ctx.device_error() == 0
+
+
+@pytest.mark.parametrize("rule", [oracle.RULE_NAIVE, oracle.RULE_MAJORITY])
+def test_tree_against_oracle(ctx, rule):
+    cfg = wl.Config("tree_s", d=256, V=4000, dtype=wl.BF16, B=3, T=0, K=8, p=0.15, kind="tree", N=25)
+    work = wl.make_workload(cfg, device=DEV)
+    cfg = work.cfg
+    ctx.set_head(work.W, max_rows=cfg.rows)
+    Wn, Hn = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H)
+    nt, npar, nh = (x.cpu().numpy() for x in (work.node_token, work.node_parent, work.node_hrow))
+    ref = oracle.verify_tree(Wn, cfg.dtype, Hn, nt, npar, nh, cfg.K, cfg.p, SEED, seq_base=2, rule=rule)
+    assert ref["accept_len"].max() >= 1          # the workload exercises accepted paths
+    for impl in _impls(ctx, cfg):
+        ctx.set_impl(impl)
+        got = to_np(ctx.verify_tree(work.H, work.node_token, work.node_parent, work.node_hrow, cfg.K, cfg.p,
+                                    SEED, seq_base=2, rule=rule))
+        ctx.set_impl(binding.IMPL_AUTO)
+        assert ctx.device_error() == 0
+        check_tree(got, ref, nt, npar, nh, rule)
+
+
+def test_host_entry_point_equals_device_entry_point(ctx):
+    cfg = wl.Config("host", d=256, V=3000, dtype=wl.BF16, B=2, T=5, K=8, p=0.1)
+    work = wl.make_workload(cfg, device=DEV)
+    ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+    dev = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=1))
+    Hh, dh = work.H.cpu().pin_memory(), work.draft.cpu().pin_memory()
+    for _ in range(2):
+        host = ctx.verify_batched_host(Hh, dh, cfg.K, cfg.p, SEED, seq_base=1)
+        for key in ("tokens", "counts", "hits", "accept_len"):
+            assert np.array_equal(host[key].numpy(), dev[key]), key
+    with pytest.raises(pk.DropMatchError) as e:
+        big = torch.zeros((cfg.B + 1, cfg.T, cfg.d), dtype=torch.bfloat16)
+        ctx.verify_batched_host(big, torch.zeros((cfg.B + 1, cfg.T), dtype=torch.int32), cfg.K, cfg.p, SEED)
+    assert e.value.status == binding.EWORKSPACE
+
+
+def test_run_to_run_determinism(ctx):
+    cfg = wl.Config("det", d=512, V=5000, dtype=wl.BF16, B=2, T=4, K=8, p=0.1)
+    work = wl.make_workload(cfg, device=DEV)
+    ctx.set_head(work.W, max_rows=cfg.rows)
+    first = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
+    for _ in range(20):
+        again = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
+        for key in first:
+            assert np.array_equal(first[key], again[key])
+
+
+def test_argument_errors(ctx):
+    cfg = wl.Config("err", d=256, V=1000, dtype=wl.BF16, B=1, T=2, K=4, p=0.1)
+    work = wl.make_workload(cfg, device=DEV)
+    fresh = pk.Context(0)
+    with pytest.raises(pk.DropMatchError) as e:
+        fresh.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED)
+    assert e.value.status == binding.ENOHEAD
+    fresh.close()
+    ctx.set_head(work.W, max_rows=cfg.rows)
+    for kw, status in ((dict(K=0), binding.EINVAL), (dict(K=2000), binding.EINVAL), (dict(p=1.0), binding.EINVAL),
+                       (dict(p=-0.1), binding.EINVAL), (dict(p=float("nan")), binding.EINVAL),
+                       (dict(rule=5), binding.EINVAL), (dict(K=16), binding.EWORKSPACE)):
+        args = dict(K=cfg.K, p=cfg.p, rule=0)
+        args.update(kw)
+        with pytest.raises(pk.DropMatchError) as e:
+            ctx.verify_batched(work.H, work.draft, args["K"], args["p"], SEED, rule=args["rule"])
+        assert e.value.status == status, kw
+    L = binding.lib()
+    assert L.dm_set_head(ctx._h, work.W.data_ptr(), 1000, 252, binding.BF16, 8, 8) == binding.EUNSUPPORTED
+    assert L.dm_set_head(ctx._h, work.W.data_ptr() + 2, 1000, 256, binding.BF16, 8, 8) == binding.EINVAL
+    # refused dm_set_head calls leave the previous head in place
+    assert ctx.workspace_bytes() > 0
+    # the context still works after the refused calls
+    ok = ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED)
+    assert int(ok["accept_len"][0]) <= cfg.T
