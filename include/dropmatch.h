@@ -17,6 +17,7 @@
  *   - Unless a parameter says "host", every tensor pointer is a DEVICE pointer on
  *     the context's device, owned by the caller, dense row-major, and must stay
  *     valid until the work queued on `stream` has finished.
+ *   - H (and W) must be 16-byte aligned (DM_EINVAL otherwise).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Device-pointer entry points only enqueue work: they never
  *     synchronise, never allocate and never free.

@@ -57,7 +57,7 @@ bool make_mask_key(float p, uint64_t seed, MaskKey* mk) {
 
 // Which kernel family serves this head under the context's override?
 int pick_impl(const dm_ctx* c, int rows, int* impl) {
-    const bool tc_ok = fused_supported(c->head, rows);
+    const bool tc_ok = c->fused != nullptr && fused_supported(c->head, rows);
     if (c->impl == DM_IMPL_TCGEN05) {
         if (!tc_ok) return DM_EUNSUPPORTED;
         *impl = DM_IMPL_TCGEN05;
@@ -96,6 +96,7 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
 
 int check_common(const dm_ctx* c, const void* H, int B, int T, int K) {
     if (c == nullptr || H == nullptr) return DM_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(H) & 15u) != 0) return DM_EINVAL;
     if (!c->has_head) return DM_ENOHEAD;
     if (B < 1 || T < 1 || K < 1 || K > kMaxK) return DM_EINVAL;
     if ((long long)B * T * K > 0x3FFFFFFFll) return DM_EINVAL;
@@ -278,6 +279,7 @@ int dropmatch_verify_tree(dm_ctx* c, const void* H, const int32_t* node_token, c
 int dm_debug_logits(dm_ctx* c, const void* H, int B, int T, const int32_t* row_sel, int n_sel, float p,
                     uint64_t seed, uint64_t seq_base, float* out_logits, void* stream) {
     if (c == nullptr || H == nullptr || row_sel == nullptr || out_logits == nullptr) return DM_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(H) & 15u) != 0) return DM_EINVAL;
     if (!c->has_head) return DM_ENOHEAD;
     if (B < 1 || T < 1 || n_sel < 1) return DM_EINVAL;
     if (n_sel > c->max_rows) return DM_EWORKSPACE;

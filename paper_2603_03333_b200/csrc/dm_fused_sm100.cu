@@ -1,10 +1,472 @@
-// placeholder: the tcgen05 kernel is added next
+// Fused sm_100a kernel for bf16 heads: Eq. 1 masks (Philox in registers), Eq. 2 masking,
+// Eq. 3 on tcgen05 tensor cores with fp32 accumulators in TMEM, and the argmax of Sec. 3.2 in
+// the epilogue, so that neither the masked hidden rows nor any logit ever reach HBM.
+//
+// Work split.  The vocabulary is cut into one contiguous slice per CTA (one CTA per SM) and
+// each slice into equal tiles of `tile_rows` <= 128 vocabulary rows.  A tile is a full
+// [tile_rows x d] strip of W, streamed exactly once through a ring of TMA stages of 64
+// hidden-size elements (128-byte swizzled rows).  The MMA is "swapped": W is the M = 128
+// operand, the masked hidden rows are the N operand (N = rows padded to a multiple of 16,
+// at most 256), so accumulator lane m is vocabulary row m of the tile and column n is path n.
+//
+// Warp roles (14 warps):
+//   warp 0      TMA producer: one thread issues cp.async.bulk.tensor loads of W
+//   warp 1      TMEM allocation; one thread issues tcgen05.mma and the commits
+//   warps 2-5   epilogue: tcgen05.ld the finished accumulator, scale by 1/(1-p), reduce each
+//               column over the 128 lanes to (max, first index), keep the best per path
+//   warps 6-13  operand builders: for every 64-element k-block write the masked hidden rows
+//               into a swizzled shared-memory ring; mask bytes come from Philox on the CTA's
+//               first tile and from a shared-memory cache on the later ones
+// Rings are guarded by mbarriers; every wait has a time limit after which the CTA sets the
+// error word, drains and frees TMEM instead of hanging.
+#include <new>
+
 #include "dm_internal.h"
+#include "dm_ptx.cuh"
+
 namespace dm {
-struct FusedState { int unused; };
-bool fused_supported(const HeadDesc&, int) { return false; }
-int fused_create(FusedState** out, const HeadDesc&, int, int, size_t* bytes) { *out = nullptr; *bytes = 0; return DM_OK; }
-void fused_destroy(FusedState*) {}
-int fused_launch(FusedState*, const HeadDesc&, const void*, int, int, const RowMap&, const MaskKey&, int*,
-                 unsigned long long*, float*, uint32_t*, cudaStream_t, int*) { return DM_EUNSUPPORTED; }
+
+namespace {
+
+constexpr int kThreads = 14 * 32;
+constexpr int kExpWarps = 8;
+constexpr int kFirstEpiWarp = 2, kFirstExpWarp = 6;
+constexpr int kBlockK = 64;                 // hidden-size elements per stage (128 bytes of bf16)
+constexpr int kTileM = 128;                 // UMMA M
+constexpr int kMaxNPad = 256;               // UMMA N limit
+constexpr int kWStageBytes = kTileM * kBlockK * 2;
+constexpr int kTmemCols = 512;
+constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
+constexpr int kSmemLimit = 227 * 1024;
+
+struct FusedParams {
+    const __nv_bfloat16* H;
+    int d, V;
+    int rows;         // paths handled by this launch (<= 256)
+    int row0;         // first path of this launch within the call
+    int rows_total;   // paths of the whole call (stride of the partials array)
+    int n_pad;        // rows rounded up to a multiple of 16
+    int kb_count;     // d / 64
+    int tiles_per_cta, tile_rows, slice_rows;
+    int nsw, nsb;     // stages of the W ring and of the operand ring
+    int cache_bits;   // keep mask bytes in shared memory after the first tile
+    RowMap map;
+    uint32_t key0, key1, thr;
+    float scale;
+    unsigned long long* partials;   // [gridDim.x][rows_total]
+    float* dbg_logits;              // [rows_total][V] or null
+    uint32_t* err;
+    // byte offsets into the 1024-aligned dynamic shared memory
+    uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar;
+};
+
+struct RowInfo { int q; uint32_t s, t, i; };
+
+__device__ __forceinline__ uint32_t mask_pair(uint32_t bits2) {
+    // bit 0 -> low bf16 kept, bit 1 -> high bf16 kept
+    return ((bits2 & 1u) ? 0x0000FFFFu : 0u) | ((bits2 & 2u) ? 0xFFFF0000u : 0u);
 }
+
+__global__ void __launch_bounds__(kThreads, 1)
+fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams P) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+    const uint32_t smem_base = ptx::smem_u32(smem);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    unsigned char* s_bits = smem + P.off_bits;
+    RowInfo* s_row = reinterpret_cast<RowInfo*>(smem + P.off_rowinfo);
+    unsigned long long* s_best = reinterpret_cast<unsigned long long*>(smem + P.off_best);  // [4][n_pad]
+    uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + P.off_bar);
+    // barrier layout: w_full[nsw] w_empty[nsw] b_ready[nsb] b_empty[nsb] acc_full[2] acc_empty[2]
+    const uint32_t bar0 = smem_base + P.off_bar;
+    const uint32_t w_full = bar0, w_empty = w_full + 8 * P.nsw;
+    const uint32_t b_ready = w_empty + 8 * P.nsw, b_empty = b_ready + 8 * P.nsb;
+    const uint32_t acc_full = b_empty + 8 * P.nsb, acc_empty = acc_full + 16;
+    const int n_bars = 2 * P.nsw + 2 * P.nsb + 4;
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + n_bars);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+    const int wps = kExpWarps / P.nsb;   // operand-builder warps per ring stage
+
+    if (threadIdx.x == 0) {
+        ptx::prefetch_tensormap(&tmap_w);
+        for (int s = 0; s < P.nsw; ++s) { ptx::mbar_init(w_full + 8 * s, 1); ptx::mbar_init(w_empty + 8 * s, 1); }
+        for (int s = 0; s < P.nsb; ++s) { ptx::mbar_init(b_ready + 8 * s, wps); ptx::mbar_init(b_empty + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { ptx::mbar_init(acc_full + 8 * s, 1); ptx::mbar_init(acc_empty + 8 * s, 4); }
+        *s_abort = 0;
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(s_tmem), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    for (int r = threadIdx.x; r < P.rows; r += kThreads) {
+        RowKey k;
+        bool ok = row_key(P.map, P.row0 + r, k);
+        if (!ok) atomicExch(P.err, (uint32_t)ERR_BAD_ROW);
+        s_row[r] = RowInfo{ok ? k.q : -1, k.s, k.t, k.i};
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    const int v_cta0 = blockIdx.x * P.slice_rows;
+    int my_tiles = 0;
+    if (v_cta0 < P.V) {
+        my_tiles = (P.V - v_cta0 + P.tile_rows - 1) / P.tile_rows;
+        if (my_tiles > P.tiles_per_cta) my_tiles = P.tiles_per_cta;
+    }
+    const int total = my_tiles * P.kb_count;   // (tile, k-block) steps of this CTA
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint32_t tx_bytes = (uint32_t)P.tile_rows * (kBlockK * 2);
+            for (int n = 0; n < total; ++n) {
+                const int s = n % P.nsw, use = n / P.nsw;
+                if (!ptx::mbar_wait(w_empty + 8 * s, (use & 1) ^ 1, s_abort, kWaitLimitCycles)) {
+                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                    break;
+                }
+                const int tile = n / P.kb_count, kb = n - tile * P.kb_count;
+                ptx::mbar_arrive_expect_tx(w_full + 8 * s, tx_bytes);
+                ptx::tma_load_2d(smem_base + P.off_w + s * kWStageBytes, &tmap_w, kb * kBlockK,
+                                 v_cta0 + tile * P.tile_rows, w_full + 8 * s);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::idesc_bf16_f32(kTileM, P.n_pad);
+            const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+            bool alive = true;
+            for (int tile = 0; tile < my_tiles && alive; ++tile) {
+                const int buf = tile & 1;
+                if (!ptx::mbar_wait(acc_empty + 8 * buf, ((tile >> 1) & 1) ^ 1, s_abort, kWaitLimitCycles)) {
+                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
+                    break;
+                }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * P.n_pad);
+                for (int kb = 0; kb < P.kb_count; ++kb) {
+                    const int n = tile * P.kb_count + kb;
+                    const int sw = n % P.nsw, sb = n % P.nsb;
+                    if (!ptx::mbar_wait(w_full + 8 * sw, (n / P.nsw) & 1, s_abort, kWaitLimitCycles)) {
+                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
+                        alive = false;
+                        break;
+                    }
+                    if (!ptx::mbar_wait(b_ready + 8 * sb, (n / P.nsb) & 1, s_abort, kWaitLimitCycles)) {
+                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
+                        alive = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint64_t a_desc = ptx::smem_desc_sw128(smem_base + P.off_w + sw * kWStageBytes);
+                    const uint64_t b_desc = ptx::smem_desc_sw128(smem_base + P.off_b + sb * b_stage_bytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
+                        ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    ptx::mma_commit(w_empty + 8 * sw);
+                    ptx::mma_commit(b_empty + 8 * sb);
+                }
+                if (alive) ptx::mma_commit(acc_full + 8 * buf);
+            }
+        }
+    } else if (warp < kFirstExpWarp) {
+        // ------------------------------------------------------------------ epilogue
+        const int ew = warp - kFirstEpiWarp;          // row of s_best owned by this warp
+        const int lane_base = (warp & 3) * 32;        // TMEM lanes this warp may read
+        unsigned long long* my_best = s_best + ew * P.n_pad;
+        for (int n = lane; n < P.n_pad; n += 32) my_best[n] = 0ull;
+        __syncwarp();
+        bool alive = true;
+        for (int tile = 0; tile < my_tiles && alive; ++tile) {
+            const int buf = tile & 1;
+            // the tcgen05.ld below needs the whole warp: make the outcome of the wait uniform
+            if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(acc_full + 8 * buf, (tile >> 1) & 1, s_abort,
+                                                        kWaitLimitCycles))) {
+                atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_FULL);
+                alive = false;
+                break;
+            }
+            ptx::tc_fence_after();
+            const int m = lane_base + lane;
+            const int v_tile0 = v_cta0 + tile * P.tile_rows;
+            const int v = v_tile0 + m;
+            const bool valid = (m < P.tile_rows) && (v < P.V);
+            const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(buf * P.n_pad);
+            for (int n0 = 0; n0 < P.n_pad; n0 += 16) {
+                uint32_t acc[16];
+                ptx::tmem_ld16(taddr + n0, acc);
+                ptx::tmem_ld_wait();
+                if (n0 + 16 >= P.n_pad) {             // accumulator fully read: hand it back
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(acc_empty + 8 * buf);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int n = n0 + j;
+                    const float val = __uint_as_float(acc[j]) * P.scale;
+                    if (P.dbg_logits != nullptr && valid && n < P.rows)
+                        P.dbg_logits[(size_t)(P.row0 + n) * P.V + v] =
+                            s_row[n].q >= 0 ? val : __uint_as_float(0x7FC00000u);
+                    const uint32_t key = valid ? float_key(val) : 0u;
+                    const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
+                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
+                    if (lane == j && mx != 0u) {
+                        const uint32_t idx = (uint32_t)(v_tile0 + lane_base + (__ffs(who) - 1));
+                        const unsigned long long cand = pack_best(mx, idx);
+                        if (cand > my_best[n]) my_best[n] = cand;
+                    }
+                }
+            }
+        }
+        ptx::bar_sync(1, 4 * 32);
+        for (int n = threadIdx.x - kFirstEpiWarp * 32; n < P.rows; n += 4 * 32) {
+            unsigned long long b = s_best[n];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) {
+                unsigned long long c = s_best[w * P.n_pad + n];
+                b = c > b ? c : b;
+            }
+            P.partials[(size_t)blockIdx.x * P.rows_total + P.row0 + n] = b;
+        }
+    } else {
+        // ------------------------------------------------------------------ operand builders
+        const int e = warp - kFirstExpWarp;
+        const int grp = e % P.nsb, sub = e / P.nsb;
+        const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+        {   // rows [rows, n_pad) of every stage stay zero for the whole kernel
+            const int tid = threadIdx.x - kFirstExpWarp * 32;
+            uint4* bz = reinterpret_cast<uint4*>(smem + P.off_b);
+            const int n16 = (int)(P.nsb * b_stage_bytes / 16);
+            for (int x = tid; x < n16; x += kExpWarps * 32) bz[x] = make_uint4(0, 0, 0, 0);
+            ptx::fence_proxy_async_smem();
+            ptx::bar_sync(2, kExpWarps * 32);
+        }
+        unsigned char* my_stage = smem + P.off_b + grp * b_stage_bytes;
+        const int n_items = P.rows * 8;            // (row, 16-byte chunk) pairs per k-block
+        const int bits_pitch = P.d >> 3;           // mask bytes per row
+        for (int n = grp; n < total; n += P.nsb) {
+            const int use = n / P.nsb;
+            if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(b_empty + 8 * grp, (use & 1) ^ 1, s_abort,
+                                                        kWaitLimitCycles))) {
+                atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                break;
+            }
+            const int tile = n / P.kb_count, kb = n - tile * P.kb_count;
+            const bool from_cache = P.cache_bits && tile > 0;
+            for (int it0 = sub * 32 + lane; it0 < n_items; it0 += 4 * wps * 32) {
+                uint4 hv[4];
+                RowInfo ri[4];
+                int r[4], c[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int it = it0 + u * wps * 32;
+                    r[u] = it >> 3; c[u] = it & 7;
+                    if (it < n_items) {
+                        ri[u] = s_row[r[u]];
+                        const int q = ri[u].q < 0 ? 0 : ri[u].q;
+                        hv[u] = __ldg(reinterpret_cast<const uint4*>(
+                            P.H + (size_t)q * P.d + kb * kBlockK + c[u] * 8));
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int it = it0 + u * wps * 32;
+                    if (it >= n_items) continue;
+                    uint32_t mbits;
+                    unsigned char* slot = s_bits + (size_t)r[u] * bits_pitch + kb * 8 + c[u];
+                    if (from_cache) {
+                        mbits = *slot;
+                    } else {
+                        RowKey k{0, ri[u].s, ri[u].t, ri[u].i};
+                        const uint32_t quad = (uint32_t)(kb * (kBlockK / 4) + c[u] * 2);
+                        mbits = keep4(quad, k, P.key0, P.key1, P.thr) |
+                                (keep4(quad + 1, k, P.key0, P.key1, P.thr) << 4);
+                        if (P.cache_bits) *slot = (unsigned char)mbits;
+                    }
+                    uint4 o;
+                    o.x = hv[u].x & mask_pair(mbits);
+                    o.y = hv[u].y & mask_pair(mbits >> 2);
+                    o.z = hv[u].z & mask_pair(mbits >> 4);
+                    o.w = hv[u].w & mask_pair(mbits >> 6);
+                    // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
+                    const uint32_t off = (uint32_t)(r[u] >> 3) * 1024u + (uint32_t)(r[u] & 7) * 128u +
+                                         (uint32_t)((c[u] ^ (r[u] & 7)) << 4);
+                    *reinterpret_cast<uint4*>(my_stage + off) = o;
+                }
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(b_ready + 8 * grp);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*s_abort) {
+        // let TMA copies that may still be in flight land before the CTA's memory is released
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------ host side
+
+struct FusedState {
+    CUtensorMap tmap_w;
+    int n_ctas, tiles_per_cta, tile_rows, slice_rows;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up at run time so that the library has no link-time
+// dependency on libcuda (it must load on machines without a driver).
+EncodeTiledFn encode_tiled_fn() {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+struct SmemPlan {
+    int nsw, nsb, cache_bits;
+    uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar, total;
+};
+
+// Split the 227 KB of shared memory between the W ring, the operand ring and the mask cache.
+bool plan_smem(int rows, int n_pad, int d, SmemPlan* out) {
+    const int kb_count = d / kBlockK;
+    const uint32_t b_stage = (uint32_t)n_pad * (kBlockK * 2);
+    const uint32_t bits = (uint32_t)rows * (uint32_t)(d / 8);
+    const uint32_t fixed = 256u * sizeof(RowInfo) + 4u * n_pad * 8u + 512u;
+    const uint32_t avail = kSmemLimit - 1024 - fixed;
+    SmemPlan best{};
+    int best_score = -1;
+    for (int cache = 1; cache >= 0; --cache)
+        for (int nsb = 8; nsb >= 2; nsb >>= 1) {
+            if (cache && (kb_count % nsb) != 0) continue;
+            const uint64_t used = (uint64_t)nsb * b_stage + (cache ? ((bits + 15u) & ~15u) : 0u);
+            if (used + 2u * kWStageBytes > avail) continue;
+            int nsw = (int)((avail - used) / kWStageBytes);
+            if (nsw > 8) nsw = 8;
+            // prefer: at least four W stages, then the mask cache, then deeper rings
+            const int score = (nsw >= 4 ? 1000 : 0) + cache * 100 + nsb * 4 + nsw;
+            if (score > best_score) {
+                best_score = score;
+                best.nsw = nsw; best.nsb = nsb; best.cache_bits = cache;
+            }
+        }
+    if (best_score < 0) return false;
+    best.off_w = 0;
+    best.off_b = (uint32_t)best.nsw * kWStageBytes;
+    best.off_bits = best.off_b + (uint32_t)best.nsb * b_stage;
+    best.off_rowinfo = best.off_bits + (best.cache_bits ? ((bits + 15u) & ~15u) : 0u);
+    best.off_best = best.off_rowinfo + 256u * sizeof(RowInfo);
+    best.off_bar = best.off_best + 4u * n_pad * 8u;
+    best.total = best.off_bar + 512u + 1024u;
+    *out = best;
+    return best.total <= (uint32_t)kSmemLimit;
+}
+
+}  // namespace
+
+bool fused_supported(const HeadDesc& head, int rows) {
+    return head.dtype == DM_BF16 && head.d >= kBlockK && head.d % kBlockK == 0 && head.V >= 1 && rows >= 1;
+}
+
+int fused_create(FusedState** out, const HeadDesc& head, int /*max_rows*/, int /*max_hidden_rows*/,
+                 size_t* bytes) {
+    *out = nullptr;
+    *bytes = 0;
+    if (!fused_supported(head, 1)) return DM_OK;   // this head runs on the CUDA-core kernel
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return DM_ECUDA;
+    FusedState* fs = new (std::nothrow) FusedState();
+    if (fs == nullptr) return DM_ECUDA;
+    int per = (head.V + sms - 1) / sms;
+    if (per < 64) per = 64;
+    fs->tiles_per_cta = (per + kTileM - 1) / kTileM;
+    fs->tile_rows = (per + fs->tiles_per_cta - 1) / fs->tiles_per_cta;
+    fs->slice_rows = fs->tiles_per_cta * fs->tile_rows;
+    fs->n_ctas = (head.V + fs->slice_rows - 1) / fs->slice_rows;
+
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (encode == nullptr) { delete fs; return DM_ECUDA; }
+    const cuuint64_t gdim[2] = {(cuuint64_t)head.d, (cuuint64_t)head.V};
+    const cuuint64_t gstride[1] = {(cuuint64_t)head.d * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)fs->tile_rows};
+    const cuuint32_t estride[2] = {1, 1};
+    CUresult r = encode(&fs->tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(head.W), gdim,
+                        gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { delete fs; return DM_ECUDA; }
+    if (cudaFuncSetAttribute(fused_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        delete fs;
+        return DM_ECUDA;
+    }
+    *out = fs;
+    return DM_OK;
+}
+
+void fused_destroy(FusedState* fs) { delete fs; }
+
+int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hidden*/, int rows,
+                 const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
+                 float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out) {
+    if (fs == nullptr || !fused_supported(head, rows) || fs->n_ctas > kMaxSlices) return DM_EUNSUPPORTED;
+    int launches = 0;
+    for (int row0 = 0; row0 < rows; row0 += kMaxNPad) {
+        FusedParams P{};
+        P.H = static_cast<const __nv_bfloat16*>(H);
+        P.d = head.d; P.V = head.V;
+        P.rows = rows - row0 < kMaxNPad ? rows - row0 : kMaxNPad;
+        P.row0 = row0; P.rows_total = rows;
+        P.n_pad = (P.rows + 15) & ~15;
+        P.kb_count = head.d / kBlockK;
+        P.tiles_per_cta = fs->tiles_per_cta; P.tile_rows = fs->tile_rows; P.slice_rows = fs->slice_rows;
+        SmemPlan plan;
+        if (!plan_smem(P.rows, P.n_pad, head.d, &plan)) return DM_EUNSUPPORTED;
+        P.nsw = plan.nsw; P.nsb = plan.nsb; P.cache_bits = plan.cache_bits;
+        P.off_w = plan.off_w; P.off_b = plan.off_b; P.off_bits = plan.off_bits;
+        P.off_rowinfo = plan.off_rowinfo; P.off_best = plan.off_best; P.off_bar = plan.off_bar;
+        P.map = map;
+        P.key0 = mk.key0; P.key1 = mk.key1; P.thr = mk.thr; P.scale = mk.scale;
+        P.partials = partials; P.dbg_logits = dbg_logits; P.err = err;
+        fused_head_kernel<<<fs->n_ctas, kThreads, plan.total, stream>>>(fs->tmap_w, P);
+        if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
+        ++launches;
+    }
+    *n_slices_out = fs->n_ctas;
+    *launches_out = launches;
+    return DM_OK;
+}
+
+}  // namespace dm
