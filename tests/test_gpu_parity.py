@@ -31,7 +31,7 @@ def _impls(ctx, cfg):
 
 def _run_chain(ctx, cfg, impl, rule=oracle.RULE_NAIVE, seq_base=0, work=None):
     work = work or wl.make_workload(cfg, device=DEV)
-    ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+    ctx.set_head(work.W, max_rows=max(cfg.rows, 16), max_hidden_rows=cfg.B * cfg.T)
     ctx.set_impl(impl)
     try:
         got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=seq_base, rule=rule))
