@@ -1,0 +1,267 @@
+#!/usr/bin/env python
+"""Benchmark of the DropMatch verification path: verify calls/s on the Llama-3-8B-shaped head.
+
+One step = one whole verify call (masked head kernel + finalize kernel) on one batch of
+synthetic input: d=4096, V=128256, bf16, T=5 draft positions, K=8 dropout paths, p=0.1, B=1.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "verify_calls_per_s"
+UNIT = "calls/s"
+WORKLOAD = "llama8b"   # Llama-3-8B-shaped head: the configuration the metric is quoted on
+
+# DRAM bytes (read + write) of one fused head-kernel launch on this workload, from the ncu capture
+# summarised in profiles/; None until a capture exists.
+NCU_TRAFFIC_BYTES = {"llama8b": None}
+
+
+def load_peaks():
+    path = ROOT / "MEASURED_PEAKS.json"
+    if path.exists():
+        p = json.loads(path.read_text())
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for (ts, r) in self.rows if (t0 is None or ts >= t0) and (t1 is None or ts <= t1 + 0.15)]
+        rows = rows or [r for (_, r) in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def time_oracle(cfg, work_cpu, steps, warmup, budget_s=20.0):
+    """Times the CPU oracle as it stands on whole verify calls; returns (calls/s, cores, sample, ms_per_step)."""
+    import oracle
+    from paper_2603_03333_b200 import workloads as wl
+    Wn, Hn = wl.to_numpy_storage(work_cpu.W), wl.to_numpy_storage(work_cpu.H)
+    draft = work_cpu.draft.numpy()
+    # a bounded sample of the call: the first `pos` draft positions (K paths each) of sequence 0
+    t0 = time.perf_counter()
+    oracle.logits_row(Wn, cfg.dtype, Hn[0, 0], cfg.p, wl.MASK_SEED, 0, 0, 0)
+    t_row = time.perf_counter() - t0
+    rows_budget = max(1, int(budget_s / max(t_row, 1e-6) / max(1, steps + warmup)))
+    pos = max(1, min(cfg.T, rows_budget // cfg.K))
+    frac = pos / (cfg.B * cfg.T)
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.verify_batched(Wn, cfg.dtype, Hn[:1, :pos], draft[:1, :pos], cfg.K, cfg.p, wl.MASK_SEED)
+        if it >= warmup:
+            times.append(time.perf_counter() - t0)
+    t_call = (sum(times) / len(times)) / frac      # scaled to the whole call (cost is linear in rows)
+    sample = (f"{pos} of {cfg.B * cfg.T} draft positions x K={cfg.K} paths per step ({pos * cfg.K} of {cfg.rows} rows), "
+              f"{len(times)} steps, scaled by rows")
+    return 1.0 / t_call, oracle.threads(), sample, t_call * 1e3
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2603_03333_b200 import workloads as wl
+    cfg = wl.CONFIGS[WORKLOAD]
+    work = wl.make_workload(cfg, device="cpu")
+    steps, warmup = max(1, min(args.steps, 3)), max(0, min(args.warmup, 1))
+    value, cores, sample, ms = time_oracle(cfg, work, steps, warmup, budget_s=60.0)
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=steps, warmup=warmup,
+                ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic",
+                config=dict(workload=WORKLOAD, d=cfg.d, V=cfg.V, B=cfg.B, T=cfg.T, K=cfg.K, p=cfg.p, rows=cfg.rows),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2603_03333_b200 as pk
+    from paper_2603_03333_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verification path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = wl.CONFIGS[args.workload]
+    work = wl.make_workload(cfg, device=dev)       # every rank: an independent replica of the call
+    ctx = pk.Context(local)
+    ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+    out = ctx.alloc_outputs(cfg.B, cfg.T, cfg.K)
+    seed = wl.MASK_SEED
+
+    def step(i):
+        ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, seed + i, out=out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin = time.perf_counter()
+    ev0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record()
+    barrier()
+    t_end = time.perf_counter()
+    clocks = sampler.stop(t_begin, t_end)
+    if ctx.device_error() != 0:
+        raise SystemExit("device error word set during the timed region")
+    ms_total = ev0.elapsed_time(ev1)
+    launches_per_step = ctx.last_launches()
+    impl_used = ctx.last_impl()
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * args.steps / (ms_total * 1e-3)
+
+    # dominant kernel alone: events on the launching stream around the head kernel of each step
+    ctx.profile_head(True)
+    for i in range(min(args.steps, 200)):
+        step(i)
+    torch.cuda.synchronize()
+    ms_sum, n_prof = ctx.profile_read()
+    ctx.profile_head(False)
+    head_ms_avg = ms_sum / max(1, n_prof)
+
+    elem = 2 if cfg.dtype == wl.BF16 else 4
+    alg_bytes = (cfg.V * cfg.d + cfg.B * cfg.T * cfg.d) * elem
+    peaks = load_peaks()
+    achieved = alg_bytes / (head_ms_avg * 1e-3) / 1e9
+    roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES.get(args.workload),
+                    kernel="fused_head_kernel", kernel_ms=head_ms_avg, algorithmic_bytes=alg_bytes,
+                    peak_source=f"of {peaks['source']} (STREAM-style copy, burst)",
+                    whole_call_gbs=alg_bytes / (ms_step * 1e-3) / 1e9)
+
+    # end to end through the host-buffer entry point: H2D of H and draft, D2H of all results, per step
+    Hh, dh = work.H.cpu().pin_memory(), work.draft.cpu().pin_memory()
+    hout = ctx.alloc_host_outputs(cfg.B, cfg.T, cfg.K)
+    for i in range(3):
+        ctx.verify_batched_host(Hh, dh, cfg.K, cfg.p, seed + i, out=hout)
+    barrier()
+    e0 = time.perf_counter()
+    n_e2e = args.steps
+    for i in range(n_e2e):
+        ctx.verify_batched_host(Hh, dh, cfg.K, cfg.p, seed + i, out=hout)   # returns after the D2H copy
+    torch.cuda.synchronize()
+    e_s = time.perf_counter() - e0
+    te = torch.tensor([e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e = dict(value=world * n_e2e / float(te.item()), unit=UNIT,
+               h2d_bytes_per_step=Hh.numel() * elem + dh.numel() * 4,
+               d2h_bytes_per_step=sum(v.numel() * 4 for v in hout.values()))
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16" if cfg.dtype == wl.BF16 else "f32", data="synthetic",
+                config=dict(workload=args.workload, d=cfg.d, V=cfg.V, B=cfg.B, T=cfg.T, K=cfg.K, p=cfg.p,
+                            rows=cfg.rows, l2="inputs larger than L2 (W is re-streamed from HBM every step)",
+                            multi_gpu="replicas only: each rank verifies its own call, no collective",
+                            impl={1: "simt", 2: "tcgen05"}.get(impl_used, "?")),
+                clocks=clocks, e2e=e2e, gpu_launches=launches_per_step * args.steps, roofline=roofline)
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        work_cpu = wl.Workload(cfg, work.W.cpu(), work.H.cpu(), work.draft.cpu(), None, None, None)
+        v, cores, sample, _ = time_oracle(cfg, work_cpu, steps=1, warmup=0, budget_s=15.0)
+        line["cpu_baseline"] = dict(value=v, unit=UNIT, cores=cores, kind="oracle", sample=sample)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -140,6 +140,15 @@ int dm_debug_masks(dm_ctx* ctx, int B, int T, int K, int d, float p, uint64_t se
  * Non-zero means a kernel abandoned an internal wait and the outputs of that call are invalid. */
 int dm_device_error(dm_ctx* ctx, void* stream, uint32_t* out_code);
 
+/* Timing of the head kernel alone (the dominant kernel).  While enabled, every verify call
+ * records a CUDA event on `stream` before and after its masked-head kernel launch(es) (not
+ * around the finalize kernel); at most 4096 calls are kept between reads, later ones are not
+ * recorded.  dm_profile_read waits for the recorded events, returns the summed elapsed time in
+ * milliseconds and the number of calls it covers, and clears the record.  Creating the events
+ * allocates driver resources, so enable it outside latency-critical code. */
+int dm_profile_head(dm_ctx* ctx, int enable);
+int dm_profile_read(dm_ctx* ctx, double* out_ms_total, int* out_calls);
+
 /* Bytes of device workspace the context holds; which kernel family the last verify call used
  * (DM_IMPL_SIMT or DM_IMPL_TCGEN05, 0 before any call); kernels launched by the last call. */
 size_t dm_workspace_bytes(const dm_ctx* ctx);

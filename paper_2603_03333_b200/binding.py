@@ -35,6 +35,8 @@ SIGNATURES = {
     "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_debug_masks": (_ci, [_vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_device_error": (_ci, [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]),
+    "dm_profile_head": (_ci, [_vp, _ci]),
+    "dm_profile_read": (_ci, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_ci)]),
     "dm_workspace_bytes": (ctypes.c_size_t, [_vp]),
     "dm_last_impl": (_ci, [_vp]),
     "dm_last_launches": (_ci, [_vp]),
@@ -207,6 +209,15 @@ class Context:
         code = ctypes.c_uint32()
         _check(lib().dm_device_error(self._h, _stream(self.device), ctypes.byref(code)), "dm_device_error")
         return code.value
+
+    def profile_head(self, enable: bool):
+        _check(lib().dm_profile_head(self._h, int(enable)), "dm_profile_head")
+
+    def profile_read(self):
+        """-> (summed head-kernel milliseconds, number of calls) since the last read."""
+        ms, n = ctypes.c_double(), ctypes.c_int()
+        _check(lib().dm_profile_read(self._h, ctypes.byref(ms), ctypes.byref(n)), "dm_profile_read")
+        return ms.value, n.value
 
     def workspace_bytes(self) -> int:
         return lib().dm_workspace_bytes(self._h)

@@ -1,6 +1,7 @@
 // C ABI of libdropmatch: argument checks, workspace, kernel choice.  See include/dropmatch.h.
 #include <math.h>
 #include <new>
+#include <vector>
 
 #include "dm_internal.h"
 
@@ -20,9 +21,15 @@ struct dm_ctx {
     int32_t* stage_i32 = nullptr;            // draft | tokens | counts | hits | accept_len
     size_t ws_bytes = 0;
     FusedState* fused = nullptr;             // tensor maps etc. of the tcgen05 kernel
+    // optional timing of the head kernel alone (dm_profile_head)
+    bool profile = false;
+    std::vector<cudaEvent_t> prof_events;    // begin/end pairs, grown on demand
+    size_t prof_used = 0;                    // events recorded since the last dm_profile_read
 };
 
 namespace {
+
+constexpr size_t kMaxProfileEvents = 8192;
 
 struct DeviceGuard {
     int prev = -1;
@@ -79,12 +86,27 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
     int st = pick_impl(c, rows, &impl);
     if (st != DM_OK) return st;
     int n_slices = 0, launches = 0;
+    cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+    if (c->profile && c->prof_used + 2 <= kMaxProfileEvents) {
+        while (c->prof_events.size() < c->prof_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+            c->prof_events.push_back(e);
+        }
+        ev_begin = c->prof_events[c->prof_used];
+        ev_end = c->prof_events[c->prof_used + 1];
+        cudaEventRecord(ev_begin, stream);
+    }
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
                           nullptr, c->err, stream, &launches);
     else {
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, stream);
         launches = 1;
+    }
+    if (ev_end != nullptr) {
+        cudaEventRecord(ev_end, stream);
+        c->prof_used += 2;
     }
     if (st != DM_OK) return st;
     st = launch_finalize(c->partials, n_slices, rows, fa, stream);
@@ -138,6 +160,7 @@ int dm_destroy(dm_ctx* c) {
     cudaDeviceSynchronize();
     free_workspace(c);
     cudaFree(c->err);
+    for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
     cudaGetLastError();
     delete c;
     return DM_OK;
@@ -329,6 +352,35 @@ int dm_device_error(dm_ctx* c, void* stream, uint32_t* out_code) {
         return DM_ECUDA;
     }
     *out_code = code;
+    return DM_OK;
+}
+
+int dm_profile_head(dm_ctx* c, int enable) {
+    if (c == nullptr) return DM_EINVAL;
+    c->profile = enable != 0;
+    return DM_OK;
+}
+
+int dm_profile_read(dm_ctx* c, double* out_ms_total, int* out_calls) {
+    if (c == nullptr || out_ms_total == nullptr || out_calls == nullptr) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    double total = 0.0;
+    int calls = 0;
+    for (size_t n = 0; n + 1 < c->prof_used; n += 2) {
+        float ms = 0.0f;
+        if (cudaEventSynchronize(c->prof_events[n + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, c->prof_events[n], c->prof_events[n + 1]) != cudaSuccess) {
+            cudaGetLastError();
+            c->prof_used = 0;
+            return DM_ECUDA;
+        }
+        total += ms;
+        ++calls;
+    }
+    c->prof_used = 0;
+    *out_ms_total = total;
+    *out_calls = calls;
     return DM_OK;
 }
 
