@@ -35,16 +35,24 @@ finalize_kernel(const unsigned long long* __restrict__ partials, int n_slices, i
     const size_t row0 = (size_t)b * TK;
 
     // split-V merge: the packed (key, inverted index) maximum over slices is the argmax with
-    // the smallest index on ties.
-    for (int x = threadIdx.x; x < TK; x += blockDim.x) {
+    // the smallest index on ties.  One warp per row: lanes stride over the slices.
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    for (int x = warp; x < TK; x += n_warps) {
         unsigned long long best = 0ull;
-        for (int s = 0; s < n_slices; ++s) {
+        for (int s = lane; s < n_slices; s += 32) {
             unsigned long long c = partials[(size_t)s * rows + row0 + x];
             best = c > best ? c : best;
         }
-        int32_t tok = (int32_t)best_index(best);
-        toks[x] = tok;
-        a.out_tokens[row0 + x] = tok;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+            best = o > best ? o : best;
+        }
+        if (lane == 0) {
+            int32_t tok = (int32_t)best_index(best);
+            toks[x] = tok;
+            a.out_tokens[row0 + x] = tok;
+        }
     }
     __syncthreads();
 

@@ -3,20 +3,26 @@
 // the epilogue, so that neither the masked hidden rows nor any logit ever reach HBM.
 //
 // Work split.  The vocabulary is cut into one contiguous slice per CTA (one CTA per SM) and
-// each slice into equal tiles of `tile_rows` <= 128 vocabulary rows.  A tile is a full
-// [tile_rows x d] strip of W, streamed exactly once through a ring of TMA stages of 64
-// hidden-size elements (128-byte swizzled rows).  The MMA is "swapped": W is the M = 128
-// operand, the masked hidden rows are the N operand (N = rows padded to a multiple of 16,
-// at most 256), so accumulator lane m is vocabulary row m of the tile and column n is path n.
+// each slice into equal tiles of `tile_rows` <= 128 vocabulary rows.  The MMA is "swapped": a
+// W tile is the M = 128 operand, the masked hidden rows are the N operand (N = rows padded to
+// a multiple of 16, at most 256), so accumulator lane m is vocabulary row m of the tile and
+// column n is path n.  TMEM (512 columns) is a ring of 512/N accumulator slots, one per tile.
+//
+// Loop order.  Tiles are taken in groups of `group_tiles`; inside a group the hidden-size
+// blocks (64 elements = one 128-byte swizzled row) are the outer loop and the tiles the inner
+// one, all accumulators of the group being live at once.  The masked operand of a block is
+// therefore built once per group (once per call when the whole slice fits in TMEM) and reused
+// by every tile of the group, while W still streams through a ring of TMA stages exactly once.
 //
 // Warp roles (14 warps):
 //   warp 0      TMA producer: one thread issues cp.async.bulk.tensor loads of W
-//   warp 1      TMEM allocation; one thread issues tcgen05.mma and the commits
-//   warps 2-5   epilogue: tcgen05.ld the finished accumulator, scale by 1/(1-p), reduce each
-//               column over the 128 lanes to (max, first index), keep the best per path
-//   warps 6-13  operand builders: for every 64-element k-block write the masked hidden rows
-//               into a swizzled shared-memory ring; mask bytes come from Philox on the CTA's
-//               first tile and from a shared-memory cache on the later ones
+//   warp 1      one thread issues tcgen05.mma and the commits
+//   warps 2-5   epilogue: tcgen05.ld a finished accumulator, scale by 1/(1-p), reduce each
+//               column over the 128 lanes to (max, first index), keep the best per path;
+//               warp 2 also allocates and frees TMEM
+//   warps 6-13  operand builders: for every (group, block) write the masked hidden rows into
+//               a swizzled shared-memory ring; mask bytes come from Philox in the first group
+//               and, when they fit, from a shared-memory cache in the later ones
 // Rings are guarded by mbarriers; every wait has a time limit after which the CTA sets the
 // error word, drains and frees TMEM instead of hanging.
 #include <new>
@@ -36,8 +42,12 @@ constexpr int kTileM = 128;                 // UMMA M
 constexpr int kMaxNPad = 256;               // UMMA N limit
 constexpr int kWStageBytes = kTileM * kBlockK * 2;
 constexpr int kTmemCols = 512;
+constexpr int kMaxWStages = 12;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
+constexpr int kPollNs = 32;                 // pause between polls of a barrier on the critical path
+constexpr int kIdlePollNs = 500;            // ... and of one that completes once per tile group
 constexpr int kSmemLimit = 227 * 1024;
+constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort flag
 
 struct FusedParams {
     const __nv_bfloat16* H;
@@ -48,8 +58,10 @@ struct FusedParams {
     int n_pad;        // rows rounded up to a multiple of 16
     int kb_count;     // d / 64
     int tiles_per_cta, tile_rows, slice_rows;
+    int group_tiles;  // tiles whose accumulators are live together
+    int n_slots;      // accumulator slots in TMEM (512 / n_pad)
     int nsw, nsb;     // stages of the W ring and of the operand ring
-    int cache_bits;   // keep mask bytes in shared memory after the first tile
+    int cache_bits;   // keep mask bytes in shared memory after the first group
     RowMap map;
     uint32_t key0, key1, thr;
     float scale;
@@ -79,12 +91,12 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
     RowInfo* s_row = reinterpret_cast<RowInfo*>(smem + P.off_rowinfo);
     unsigned long long* s_best = reinterpret_cast<unsigned long long*>(smem + P.off_best);  // [4][n_pad]
     uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + P.off_bar);
-    // barrier layout: w_full[nsw] w_empty[nsw] b_ready[nsb] b_empty[nsb] acc_full[2] acc_empty[2]
+    // barrier layout: w_full[nsw] w_empty[nsw] b_ready[nsb] b_empty[nsb] slot_full[S] slot_empty[S]
     const uint32_t bar0 = smem_base + P.off_bar;
     const uint32_t w_full = bar0, w_empty = w_full + 8 * P.nsw;
     const uint32_t b_ready = w_empty + 8 * P.nsw, b_empty = b_ready + 8 * P.nsb;
-    const uint32_t acc_full = b_empty + 8 * P.nsb, acc_empty = acc_full + 16;
-    const int n_bars = 2 * P.nsw + 2 * P.nsb + 4;
+    const uint32_t slot_full = b_empty + 8 * P.nsb, slot_empty = slot_full + 8 * P.n_slots;
+    const int n_bars = 2 * P.nsw + 2 * P.nsb + 2 * P.n_slots;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + n_bars);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
@@ -94,12 +106,12 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         ptx::prefetch_tensormap(&tmap_w);
         for (int s = 0; s < P.nsw; ++s) { ptx::mbar_init(w_full + 8 * s, 1); ptx::mbar_init(w_empty + 8 * s, 1); }
         for (int s = 0; s < P.nsb; ++s) { ptx::mbar_init(b_ready + 8 * s, wps); ptx::mbar_init(b_empty + 8 * s, 1); }
-        for (int s = 0; s < 2; ++s) { ptx::mbar_init(acc_full + 8 * s, 1); ptx::mbar_init(acc_empty + 8 * s, 4); }
+        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, 4); }
         *s_abort = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
     }
-    if (warp == 1) {
+    if (warp == kFirstEpiWarp) {   // an epilogue warp owns TMEM: it is still whole at the end
         ptx::tmem_alloc(ptx::smem_u32(s_tmem), kTmemCols);
         ptx::tmem_relinquish();
     }
@@ -120,63 +132,75 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         my_tiles = (P.V - v_cta0 + P.tile_rows - 1) / P.tile_rows;
         if (my_tiles > P.tiles_per_cta) my_tiles = P.tiles_per_cta;
     }
-    const int total = my_tiles * P.kb_count;   // (tile, k-block) steps of this CTA
+    const int G = P.group_tiles;
+    const int n_groups = (my_tiles + G - 1) / G;
 
+    // Polling an mbarrier is not free for the TMA unit that updates it, so each wait is made by
+    // one lane only.  The producer and the MMA issuer are single threads; the other lanes of
+    // their warps retire at once instead of idling at a barrier.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            const uint32_t tx_bytes = (uint32_t)P.tile_rows * (kBlockK * 2);
-            for (int n = 0; n < total; ++n) {
-                const int s = n % P.nsw, use = n / P.nsw;
-                if (!ptx::mbar_wait(w_empty + 8 * s, (use & 1) ^ 1, s_abort, kWaitLimitCycles)) {
-                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
-                    break;
+        if (lane != 0) return;
+        const uint32_t tx_bytes = (uint32_t)P.tile_rows * (kBlockK * 2);
+        int n = 0;
+        for (int g = 0; g < n_groups; ++g) {
+            const int t0 = g * G, t1 = min(my_tiles, t0 + G);
+            for (int kb = 0; kb < P.kb_count; ++kb)
+                for (int tile = t0; tile < t1; ++tile, ++n) {
+                    const int s = n % P.nsw, use = n / P.nsw;
+                    if (!ptx::mbar_wait<kPollNs>(w_empty + 8 * s, (use & 1) ^ 1, s_abort, kWaitLimitCycles)) {
+                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                        return;
+                    }
+                    ptx::mbar_arrive_expect_tx(w_full + 8 * s, tx_bytes);
+                    ptx::tma_load_2d(smem_base + P.off_w + s * kWStageBytes, &tmap_w, kb * kBlockK,
+                                     v_cta0 + tile * P.tile_rows, w_full + 8 * s);
                 }
-                const int tile = n / P.kb_count, kb = n - tile * P.kb_count;
-                ptx::mbar_arrive_expect_tx(w_full + 8 * s, tx_bytes);
-                ptx::tma_load_2d(smem_base + P.off_w + s * kWStageBytes, &tmap_w, kb * kBlockK,
-                                 v_cta0 + tile * P.tile_rows, w_full + 8 * s);
-            }
         }
+        return;
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = ptx::idesc_bf16_f32(kTileM, P.n_pad);
-            const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
-            bool alive = true;
-            for (int tile = 0; tile < my_tiles && alive; ++tile) {
-                const int buf = tile & 1;
-                if (!ptx::mbar_wait(acc_empty + 8 * buf, ((tile >> 1) & 1) ^ 1, s_abort, kWaitLimitCycles)) {
+        if (lane != 0) return;
+        const uint32_t idesc = ptx::idesc_bf16_f32(kTileM, P.n_pad);
+        const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+        int n = 0, m = 0;   // W-ring step, operand-ring step
+        for (int g = 0; g < n_groups; ++g) {
+            const int t0 = g * G, t1 = min(my_tiles, t0 + G);
+            for (int tile = t0; tile < t1; ++tile) {   // the group's accumulator slots must be drained
+                const int slot = tile % P.n_slots;
+                if (!ptx::mbar_wait<kPollNs>(slot_empty + 8 * slot, ((tile / P.n_slots) & 1) ^ 1, s_abort,
+                                             kWaitLimitCycles)) {
                     atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
-                    break;
+                    return;
                 }
-                ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * P.n_pad);
-                for (int kb = 0; kb < P.kb_count; ++kb) {
-                    const int n = tile * P.kb_count + kb;
-                    const int sw = n % P.nsw, sb = n % P.nsb;
-                    if (!ptx::mbar_wait(w_full + 8 * sw, (n / P.nsw) & 1, s_abort, kWaitLimitCycles)) {
+            }
+            ptx::tc_fence_after();
+            for (int kb = 0; kb < P.kb_count; ++kb, ++m) {
+                const int sb = m % P.nsb;
+                if (!ptx::mbar_wait<kPollNs>(b_ready + 8 * sb, (m / P.nsb) & 1, s_abort, kWaitLimitCycles)) {
+                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
+                    return;
+                }
+                const uint64_t b_desc = ptx::smem_desc_sw128(smem_base + P.off_b + sb * b_stage_bytes);
+                for (int tile = t0; tile < t1; ++tile, ++n) {
+                    const int sw = n % P.nsw;
+                    if (!ptx::mbar_wait<kPollNs>(w_full + 8 * sw, (n / P.nsw) & 1, s_abort, kWaitLimitCycles)) {
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
-                        alive = false;
-                        break;
-                    }
-                    if (!ptx::mbar_wait(b_ready + 8 * sb, (n / P.nsb) & 1, s_abort, kWaitLimitCycles)) {
-                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
-                        alive = false;
-                        break;
+                        return;
                     }
                     ptx::tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)((tile % P.n_slots) * P.n_pad);
                     const uint64_t a_desc = ptx::smem_desc_sw128(smem_base + P.off_w + sw * kWStageBytes);
-                    const uint64_t b_desc = ptx::smem_desc_sw128(smem_base + P.off_b + sb * b_stage_bytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
                         ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
                     ptx::mma_commit(w_empty + 8 * sw);
-                    ptx::mma_commit(b_empty + 8 * sb);
                 }
-                if (alive) ptx::mma_commit(acc_full + 8 * buf);
+                ptx::mma_commit(b_empty + 8 * sb);
             }
+            for (int tile = t0; tile < t1; ++tile) ptx::mma_commit(slot_full + 8 * (tile % P.n_slots));
         }
+        return;
     } else if (warp < kFirstExpWarp) {
         // ------------------------------------------------------------------ epilogue
         const int ew = warp - kFirstEpiWarp;          // row of s_best owned by this warp
@@ -186,10 +210,10 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         __syncwarp();
         bool alive = true;
         for (int tile = 0; tile < my_tiles && alive; ++tile) {
-            const int buf = tile & 1;
-            // the tcgen05.ld below needs the whole warp: make the outcome of the wait uniform
-            if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(acc_full + 8 * buf, (tile >> 1) & 1, s_abort,
-                                                        kWaitLimitCycles))) {
+            const int slot = tile % P.n_slots;
+            // the tcgen05.ld below needs the whole warp: the outcome of the wait is warp-uniform
+            if (!ptx::mbar_wait_warp<kIdlePollNs>(slot_full + 8 * slot, (tile / P.n_slots) & 1, s_abort,
+                                                  kWaitLimitCycles)) {
                 atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_FULL);
                 alive = false;
                 break;
@@ -199,15 +223,15 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
             const int v_tile0 = v_cta0 + tile * P.tile_rows;
             const int v = v_tile0 + m;
             const bool valid = (m < P.tile_rows) && (v < P.V);
-            const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(buf * P.n_pad);
+            const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(slot * P.n_pad);
             for (int n0 = 0; n0 < P.n_pad; n0 += 16) {
                 uint32_t acc[16];
                 ptx::tmem_ld16(taddr + n0, acc);
                 ptx::tmem_ld_wait();
-                if (n0 + 16 >= P.n_pad) {             // accumulator fully read: hand it back
+                if (n0 + 16 >= P.n_pad) {             // accumulator fully read: hand the slot back
                     ptx::tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(acc_empty + 8 * buf);
+                    if (lane == 0) ptx::mbar_arrive(slot_empty + 8 * slot);
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
@@ -237,6 +261,17 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
             }
             P.partials[(size_t)blockIdx.x * P.rows_total + P.row0 + n] = b;
         }
+        // ------------------------------------------------------------------ teardown
+        // Every accumulator has been read, hence every MMA and every TMA load has completed.
+        // After an abandoned wait, give copies that may still be in flight time to land first.
+        if (*s_abort)
+            for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        ptx::tc_fence_before();
+        ptx::bar_sync(1, 4 * 32);
+        if (warp == kFirstEpiWarp) {
+            ptx::tc_fence_after();
+            ptx::tmem_dealloc(tmem_base, kTmemCols);
+        }
     } else {
         // ------------------------------------------------------------------ operand builders
         const int e = warp - kFirstExpWarp;
@@ -251,43 +286,54 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
             ptx::bar_sync(2, kExpWarps * 32);
         }
         unsigned char* my_stage = smem + P.off_b + grp * b_stage_bytes;
-        const int n_items = P.rows * 8;            // (row, 16-byte chunk) pairs per k-block
+        const int n_items = P.rows * 8;            // (row, 16-byte chunk) pairs per block
         const int bits_pitch = P.d >> 3;           // mask bytes per row
-        for (int n = grp; n < total; n += P.nsb) {
-            const int use = n / P.nsb;
-            if (!__all_sync(0xFFFFFFFFu, ptx::mbar_wait(b_empty + 8 * grp, (use & 1) ^ 1, s_abort,
-                                                        kWaitLimitCycles))) {
+        const int stride = wps * 32;               // threads working on this stage
+        const int total_b = n_groups * P.kb_count;
+        for (int m = grp; m < total_b; m += P.nsb) {
+            const int g = m / P.kb_count, kb = m - g * P.kb_count;
+            const bool from_cache = P.cache_bits && g > 0;
+            const __nv_bfloat16* h_kb = P.H + kb * kBlockK;
+            // the hidden-state loads do not depend on the stage being free: start them first
+            uint4 hv[4];
+            int it0 = sub * 32 + lane;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int it = it0 + u * stride;
+                if (it < n_items) {
+                    const int q = max(s_row[it >> 3].q, 0);
+                    hv[u] = __ldg(reinterpret_cast<const uint4*>(h_kb + (size_t)q * P.d + (it & 7) * 8));
+                }
+            }
+            if (!ptx::mbar_wait_warp<kPollNs>(b_empty + 8 * grp, ((m / P.nsb) & 1) ^ 1, s_abort,
+                                              kWaitLimitCycles)) {
                 atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                 break;
             }
-            const int tile = n / P.kb_count, kb = n - tile * P.kb_count;
-            const bool from_cache = P.cache_bits && tile > 0;
-            for (int it0 = sub * 32 + lane; it0 < n_items; it0 += 4 * wps * 32) {
-                uint4 hv[4];
-                RowInfo ri[4];
-                int r[4], c[4];
+            for (; it0 < n_items; it0 += 4 * stride) {
+                // next batch of hidden-state chunks, in flight while this batch is masked
+                uint4 hv_next[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int it = it0 + u * wps * 32;
-                    r[u] = it >> 3; c[u] = it & 7;
+                    const int it = it0 + (4 + u) * stride;
                     if (it < n_items) {
-                        ri[u] = s_row[r[u]];
-                        const int q = ri[u].q < 0 ? 0 : ri[u].q;
-                        hv[u] = __ldg(reinterpret_cast<const uint4*>(
-                            P.H + (size_t)q * P.d + kb * kBlockK + c[u] * 8));
+                        const int q = max(s_row[it >> 3].q, 0);
+                        hv_next[u] = __ldg(reinterpret_cast<const uint4*>(h_kb + (size_t)q * P.d + (it & 7) * 8));
                     }
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int it = it0 + u * wps * 32;
+                    const int it = it0 + u * stride;
                     if (it >= n_items) continue;
+                    const int r = it >> 3, c = it & 7;
                     uint32_t mbits;
-                    unsigned char* slot = s_bits + (size_t)r[u] * bits_pitch + kb * 8 + c[u];
+                    unsigned char* slot = s_bits + (size_t)r * bits_pitch + kb * 8 + c;
                     if (from_cache) {
                         mbits = *slot;
                     } else {
-                        RowKey k{0, ri[u].s, ri[u].t, ri[u].i};
-                        const uint32_t quad = (uint32_t)(kb * (kBlockK / 4) + c[u] * 2);
+                        const RowInfo ri = s_row[r];
+                        RowKey k{0, ri.s, ri.t, ri.i};
+                        const uint32_t quad = (uint32_t)(kb * (kBlockK / 4) + c * 2);
                         mbits = keep4(quad, k, P.key0, P.key1, P.thr) |
                                 (keep4(quad + 1, k, P.key0, P.key1, P.thr) << 4);
                         if (P.cache_bits) *slot = (unsigned char)mbits;
@@ -298,10 +344,12 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
                     o.z = hv[u].z & mask_pair(mbits >> 4);
                     o.w = hv[u].w & mask_pair(mbits >> 6);
                     // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
-                    const uint32_t off = (uint32_t)(r[u] >> 3) * 1024u + (uint32_t)(r[u] & 7) * 128u +
-                                         (uint32_t)((c[u] ^ (r[u] & 7)) << 4);
+                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u +
+                                         (uint32_t)((c ^ (r & 7)) << 4);
                     *reinterpret_cast<uint4*>(my_stage + off) = o;
                 }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) hv[u] = hv_next[u];
             }
             ptx::fence_proxy_async_smem();
             __syncwarp();
@@ -309,18 +357,6 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         }
     }
 
-    // ---------------------------------------------------------------------- teardown
-    if (*s_abort) {
-        // let TMA copies that may still be in flight land before the CTA's memory is released
-        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        __syncwarp();
-        ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
-    }
 }
 
 }  // namespace
@@ -353,28 +389,40 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 struct SmemPlan {
-    int nsw, nsb, cache_bits;
+    int nsw, nsb, cache_bits, group_tiles, n_slots;
     uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar, total;
 };
 
-// Split the 227 KB of shared memory between the W ring, the operand ring and the mask cache.
-bool plan_smem(int rows, int n_pad, int d, SmemPlan* out) {
+// Choose the tile grouping, then split the 227 KB of shared memory between the W ring, the
+// operand ring and (only when tiles need more than one group) the mask cache.
+bool plan_smem(int rows, int n_pad, int d, int tiles_per_cta, SmemPlan* out) {
+    SmemPlan best{};
+    best.n_slots = kTmemCols / n_pad;
+    if (tiles_per_cta <= best.n_slots) {
+        best.group_tiles = tiles_per_cta;               // the whole slice is live at once
+    } else {
+        // several groups: use half of the slots per group so that the epilogue of one group
+        // overlaps the MMAs of the next, and even the group sizes out
+        int g = best.n_slots / 2 > 0 ? best.n_slots / 2 : 1;
+        const int n_groups = (tiles_per_cta + g - 1) / g;
+        best.group_tiles = (tiles_per_cta + n_groups - 1) / n_groups;
+    }
+    const bool multi = best.group_tiles < tiles_per_cta;
     const int kb_count = d / kBlockK;
     const uint32_t b_stage = (uint32_t)n_pad * (kBlockK * 2);
-    const uint32_t bits = (uint32_t)rows * (uint32_t)(d / 8);
-    const uint32_t fixed = 256u * sizeof(RowInfo) + 4u * n_pad * 8u + 512u;
+    const uint32_t bits = ((uint32_t)rows * (uint32_t)(d / 8) + 15u) & ~15u;
+    const uint32_t fixed = 256u * sizeof(RowInfo) + 4u * n_pad * 8u + kBarBytes;
     const uint32_t avail = kSmemLimit - 1024 - fixed;
-    SmemPlan best{};
     int best_score = -1;
-    for (int cache = 1; cache >= 0; --cache)
-        for (int nsb = 8; nsb >= 2; nsb >>= 1) {
+    for (int cache = multi ? 1 : 0; cache >= 0; --cache)
+        for (int nsb = 4; nsb >= 2; nsb >>= 1) {
             if (cache && (kb_count % nsb) != 0) continue;
-            const uint64_t used = (uint64_t)nsb * b_stage + (cache ? ((bits + 15u) & ~15u) : 0u);
+            const uint64_t used = (uint64_t)nsb * b_stage + (cache ? bits : 0u);
             if (used + 2u * kWStageBytes > avail) continue;
             int nsw = (int)((avail - used) / kWStageBytes);
-            if (nsw > 8) nsw = 8;
-            // prefer: at least four W stages, then the mask cache, then deeper rings
-            const int score = (nsw >= 4 ? 1000 : 0) + cache * 100 + nsb * 4 + nsw;
+            if (nsw > kMaxWStages) nsw = kMaxWStages;
+            // prefer: at least six W stages, then the mask cache, then deeper rings
+            const int score = (nsw >= 6 ? 1000 : 0) + cache * 100 + nsb * 4 + nsw;
             if (score > best_score) {
                 best_score = score;
                 best.nsw = nsw; best.nsb = nsb; best.cache_bits = cache;
@@ -384,10 +432,10 @@ bool plan_smem(int rows, int n_pad, int d, SmemPlan* out) {
     best.off_w = 0;
     best.off_b = (uint32_t)best.nsw * kWStageBytes;
     best.off_bits = best.off_b + (uint32_t)best.nsb * b_stage;
-    best.off_rowinfo = best.off_bits + (best.cache_bits ? ((bits + 15u) & ~15u) : 0u);
+    best.off_rowinfo = best.off_bits + (best.cache_bits ? bits : 0u);
     best.off_best = best.off_rowinfo + 256u * sizeof(RowInfo);
     best.off_bar = best.off_best + 4u * n_pad * 8u;
-    best.total = best.off_bar + 512u + 1024u;
+    best.total = best.off_bar + kBarBytes + 1024u;
     *out = best;
     return best.total <= (uint32_t)kSmemLimit;
 }
@@ -453,7 +501,8 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.kb_count = head.d / kBlockK;
         P.tiles_per_cta = fs->tiles_per_cta; P.tile_rows = fs->tile_rows; P.slice_rows = fs->slice_rows;
         SmemPlan plan;
-        if (!plan_smem(P.rows, P.n_pad, head.d, &plan)) return DM_EUNSUPPORTED;
+        if (!plan_smem(P.rows, P.n_pad, head.d, fs->tiles_per_cta, &plan)) return DM_EUNSUPPORTED;
+        P.group_tiles = plan.group_tiles; P.n_slots = plan.n_slots;
         P.nsw = plan.nsw; P.nsb = plan.nsb; P.cache_bits = plan.cache_bits;
         P.off_w = plan.off_w; P.off_b = plan.off_b; P.off_bits = plan.off_bits;
         P.off_rowinfo = plan.off_rowinfo; P.off_best = plan.off_best; P.off_bar = plan.off_bar;

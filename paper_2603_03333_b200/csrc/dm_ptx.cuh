@@ -22,6 +22,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One try: the hardware may suspend the thread for a short, system-dependent time while the
+// phase with this parity has not completed.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t done;
     asm volatile(
@@ -41,18 +43,30 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 
 // Wait with a time limit.  Returns false if the limit ran out or another thread already gave
 // up (abort flag in shared memory); the caller then leaves its loop and the CTA tears down.
+// Polling an mbarrier competes with the TMA unit that updates it, so only one lane of a warp
+// should call this, and a waiter that is not on the critical path sleeps SLEEP_NS between tries.
+template <int SLEEP_NS>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
+    for (;;) {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+        if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             return false;
         }
     }
-    return true;
+}
+// The same wait for a whole warp: lane 0 polls, the other lanes pick the outcome up.
+template <int SLEEP_NS>
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               long long limit_cycles) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait<SLEEP_NS>(bar, parity, abort_flag, limit_cycles) ? 1 : 0;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 
 // ---- TMA ----------------------------------------------------------------------------------

@@ -76,6 +76,11 @@ SMALL = [
     wl.Config("f32_b", d=100, V=517, dtype=wl.F32, B=2, T=3, K=7, p=0.2, draft_mode="toy"),
     wl.Config("bf16_rows200", d=256, V=2500, dtype=wl.BF16, B=5, T=5, K=8, p=0.1),
     wl.Config("bf16_rows300", d=128, V=1500, dtype=wl.BF16, B=3, T=10, K=10, p=0.1),
+    # vocabulary slices of several tiles per CTA whose accumulators do not all fit in TMEM at once:
+    # four groups of one tile with the mask cache, two groups of two tiles, three groups without cache
+    wl.Config("bf16_groups4", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1),
+    wl.Config("bf16_groups2", d=256, V=61111, dtype=wl.BF16, B=2, T=4, K=16, p=0.2),
+    wl.Config("bf16_groups_nocache", d=192, V=50000, dtype=wl.BF16, B=1, T=9, K=16, p=0.1),
 ]
 
 
