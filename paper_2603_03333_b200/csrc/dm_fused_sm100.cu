@@ -205,9 +205,12 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         // ------------------------------------------------------------------ epilogue
         const int ew = warp - kFirstEpiWarp;          // row of s_best owned by this warp
         const int lane_base = (warp & 3) * 32;        // TMEM lanes this warp may read
-        unsigned long long* my_best = s_best + ew * P.n_pad;
-        for (int n = lane; n < P.n_pad; n += 32) my_best[n] = 0ull;
-        __syncwarp();
+        // Columns are taken 16 at a time.  Column 16*c + j is owned by lane j (c even) or lane
+        // 16 + j (c odd), which keeps that path's running best (key, index) in registers
+        // across all tiles; nothing is exchanged through shared memory until the end.
+        uint32_t best_key[kMaxNPad / 32], best_idx[kMaxNPad / 32];
+#pragma unroll
+        for (int c2 = 0; c2 < kMaxNPad / 32; ++c2) { best_key[c2] = 0u; best_idx[c2] = 0u; }
         bool alive = true;
         for (int tile = 0; tile < my_tiles && alive; ++tile) {
             const int slot = tile % P.n_slots;
@@ -224,32 +227,46 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
             const int v = v_tile0 + m;
             const bool valid = (m < P.tile_rows) && (v < P.V);
             const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(slot * P.n_pad);
-            for (int n0 = 0; n0 < P.n_pad; n0 += 16) {
-                uint32_t acc[16];
-                ptx::tmem_ld16(taddr + n0, acc);
-                ptx::tmem_ld_wait();
-                if (n0 + 16 >= P.n_pad) {             // accumulator fully read: hand the slot back
-                    ptx::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(slot_empty + 8 * slot);
-                }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int n = n0 + j;
-                    const float val = __uint_as_float(acc[j]) * P.scale;
-                    if (P.dbg_logits != nullptr && valid && n < P.rows)
-                        P.dbg_logits[(size_t)(P.row0 + n) * P.V + v] =
-                            s_row[n].q >= 0 ? val : __uint_as_float(0x7FC00000u);
-                    const uint32_t key = valid ? float_key(val) : 0u;
-                    const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
-                    if (lane == j && mx != 0u) {
-                        const uint32_t idx = (uint32_t)(v_tile0 + lane_base + (__ffs(who) - 1));
-                        const unsigned long long cand = pack_best(mx, idx);
-                        if (cand > my_best[n]) my_best[n] = cand;
+            for (int c = 0; c < kMaxNPad / 16; ++c) {
+                const int n0 = c * 16;
+                if (n0 < P.n_pad) {
+                    uint32_t acc[16];
+                    ptx::tmem_ld16(taddr + n0, acc);
+                    ptx::tmem_ld_wait();
+                    if (n0 + 16 >= P.n_pad) {             // accumulator fully read: hand the slot back
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(slot_empty + 8 * slot);
+                    }
+                    uint32_t cur_key = 0u, cur_who = 0u;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float val = __uint_as_float(acc[j]) * P.scale;
+                        if (P.dbg_logits != nullptr && valid && n0 + j < P.rows)
+                            P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
+                                s_row[n0 + j].q >= 0 ? val : __uint_as_float(0x7FC00000u);
+                        const uint32_t key = valid ? float_key(val) : 0u;
+                        const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
+                        const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
+                        const bool mine = lane == (c & 1) * 16 + j;
+                        cur_key = mine ? mx : cur_key;
+                        cur_who = mine ? who : cur_who;
+                    }
+                    // a later tile holds larger indices, so only a strictly larger key replaces
+                    if (cur_key > best_key[c >> 1]) {
+                        best_key[c >> 1] = cur_key;
+                        best_idx[c >> 1] = (uint32_t)(v_tile0 + lane_base + (__ffs(cur_who) - 1));
                     }
                 }
             }
+        }
+        unsigned long long* my_best = s_best + ew * P.n_pad;
+#pragma unroll
+        for (int c = 0; c < kMaxNPad / 16; ++c) {
+            const int n = c * 16 + (lane & 15);
+            if (n < P.n_pad && (lane >> 4) == (c & 1))
+                my_best[n] = best_key[c >> 1] != 0u ? pack_best(best_key[c >> 1], best_idx[c >> 1]) : 0ull;
         }
         ptx::bar_sync(1, 4 * 32);
         for (int n = threadIdx.x - kFirstEpiWarp * 32; n < P.rows; n += 4 * 32) {
