@@ -17,9 +17,9 @@
 // Warp roles (14 warps):
 //   warp 0      TMA producer: one thread issues cp.async.bulk.tensor loads of W
 //   warp 1      one thread issues tcgen05.mma and the commits
-//   warps 2-5   epilogue: tcgen05.ld a finished accumulator, scale by 1/(1-p), reduce each
-//               column over the 128 lanes to (max, first index), keep the best per path;
-//               warp 2 also allocates and frees TMEM
+//   warps 2-5   epilogue: tcgen05.ld the finished accumulators of a group, scale by 1/(1-p),
+//               reduce each column over tiles and lanes to (max, first index), keep the best
+//               per path; warp 2 also allocates and frees TMEM
 //   warps 6-13  operand builders: for every (group, block) write the masked hidden rows into
 //               a swizzled shared-memory ring; mask bytes come from Philox in the first group
 //               and, when they fit, from a shared-memory cache in the later ones
@@ -141,21 +141,30 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane != 0) return;
+        // Ring positions, phases and coordinates advance by increments: this lone thread must
+        // issue one load every few hundred cycles, and an integer division costs about that.
         const uint32_t tx_bytes = (uint32_t)P.tile_rows * (kBlockK * 2);
-        int n = 0;
+        uint32_t bar_full = w_full, bar_empty = w_empty, dst = smem_base + P.off_w, empty_parity = 1;
+        int stage = 0;
         for (int g = 0; g < n_groups; ++g) {
             const int t0 = g * G, t1 = min(my_tiles, t0 + G);
-            for (int kb = 0; kb < P.kb_count; ++kb)
-                for (int tile = t0; tile < t1; ++tile, ++n) {
-                    const int s = n % P.nsw, use = n / P.nsw;
-                    if (!ptx::mbar_wait<kPollNs>(w_empty + 8 * s, (use & 1) ^ 1, s_abort, kWaitLimitCycles)) {
+            const int v_first = v_cta0 + t0 * P.tile_rows;
+            for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
+                int v_tile = v_first;
+                for (int tile = t0; tile < t1; ++tile, v_tile += P.tile_rows) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_empty, empty_parity, s_abort, kWaitLimitCycles)) {
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                         return;
                     }
-                    ptx::mbar_arrive_expect_tx(w_full + 8 * s, tx_bytes);
-                    ptx::tma_load_2d(smem_base + P.off_w + s * kWStageBytes, &tmap_w, kb * kBlockK,
-                                     v_cta0 + tile * P.tile_rows, w_full + 8 * s);
+                    ptx::mbar_arrive_expect_tx(bar_full, tx_bytes);
+                    ptx::tma_load_2d(dst, &tmap_w, x, v_tile, bar_full);
+                    bar_full += 8; bar_empty += 8; dst += kWStageBytes;
+                    if (++stage == P.nsw) {
+                        stage = 0; empty_parity ^= 1;
+                        bar_full = w_full; bar_empty = w_empty; dst = smem_base + P.off_w;
+                    }
                 }
+            }
         }
         return;
     } else if (warp == 1) {
@@ -163,100 +172,136 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         if (lane != 0) return;
         const uint32_t idesc = ptx::idesc_bf16_f32(kTileM, P.n_pad);
         const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
-        int n = 0, m = 0;   // W-ring step, operand-ring step
+        const uint64_t a_desc0 = ptx::smem_desc_sw128(smem_base + P.off_w);
+        const uint64_t b_desc0 = ptx::smem_desc_sw128(smem_base + P.off_b);
+        // W ring, operand ring and accumulator-slot cursors, all advanced by increments
+        int sw = 0, sb = 0, slot = 0;
+        uint32_t w_parity = 0, b_parity = 0, slot_parity = 1;   // slot_parity: parity of the slot_empty wait
+        uint64_t a_desc = a_desc0, b_desc = b_desc0;
+        uint32_t bar_wf = w_full, bar_we = w_empty, bar_br = b_ready, bar_be = b_empty;
         for (int g = 0; g < n_groups; ++g) {
             const int t0 = g * G, t1 = min(my_tiles, t0 + G);
+            const int slot0 = slot;
             for (int tile = t0; tile < t1; ++tile) {   // the group's accumulator slots must be drained
-                const int slot = tile % P.n_slots;
-                if (!ptx::mbar_wait<kPollNs>(slot_empty + 8 * slot, ((tile / P.n_slots) & 1) ^ 1, s_abort,
-                                             kWaitLimitCycles)) {
+                if (!ptx::mbar_wait<kPollNs>(slot_empty + 8 * slot, slot_parity, s_abort, kWaitLimitCycles)) {
                     atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
                     return;
                 }
+                if (++slot == P.n_slots) { slot = 0; slot_parity ^= 1; }
             }
             ptx::tc_fence_after();
-            for (int kb = 0; kb < P.kb_count; ++kb, ++m) {
-                const int sb = m % P.nsb;
-                if (!ptx::mbar_wait<kPollNs>(b_ready + 8 * sb, (m / P.nsb) & 1, s_abort, kWaitLimitCycles)) {
+            for (int kb = 0; kb < P.kb_count; ++kb) {
+                if (!ptx::mbar_wait<kPollNs>(bar_br, b_parity, s_abort, kWaitLimitCycles)) {
                     atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
                     return;
                 }
-                const uint64_t b_desc = ptx::smem_desc_sw128(smem_base + P.off_b + sb * b_stage_bytes);
-                for (int tile = t0; tile < t1; ++tile, ++n) {
-                    const int sw = n % P.nsw;
-                    if (!ptx::mbar_wait<kPollNs>(w_full + 8 * sw, (n / P.nsw) & 1, s_abort, kWaitLimitCycles)) {
+                int sl = slot0;
+                uint32_t d_tmem = tmem_base + (uint32_t)(slot0 * P.n_pad);
+                for (int tile = t0; tile < t1; ++tile) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_wf, w_parity, s_abort, kWaitLimitCycles)) {
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
                         return;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)((tile % P.n_slots) * P.n_pad);
-                    const uint64_t a_desc = ptx::smem_desc_sw128(smem_base + P.off_w + sw * kWStageBytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
                         ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-                    ptx::mma_commit(w_empty + 8 * sw);
+                    ptx::mma_commit(bar_we);
+                    bar_wf += 8; bar_we += 8; a_desc += kWStageBytes >> 4;
+                    if (++sw == P.nsw) { sw = 0; w_parity ^= 1; bar_wf = w_full; bar_we = w_empty; a_desc = a_desc0; }
+                    d_tmem += (uint32_t)P.n_pad;
+                    if (++sl == P.n_slots) { sl = 0; d_tmem = tmem_base; }
                 }
-                ptx::mma_commit(b_empty + 8 * sb);
+                ptx::mma_commit(bar_be);
+                bar_br += 8; bar_be += 8; b_desc += b_stage_bytes >> 4;
+                if (++sb == P.nsb) { sb = 0; b_parity ^= 1; bar_br = b_ready; bar_be = b_empty; b_desc = b_desc0; }
             }
-            for (int tile = t0; tile < t1; ++tile) ptx::mma_commit(slot_full + 8 * (tile % P.n_slots));
+            int sl = slot0;
+            for (int tile = t0; tile < t1; ++tile) {
+                ptx::mma_commit(slot_full + 8 * sl);
+                if (++sl == P.n_slots) sl = 0;
+            }
         }
         return;
     } else if (warp < kFirstExpWarp) {
         // ------------------------------------------------------------------ epilogue
         const int ew = warp - kFirstEpiWarp;          // row of s_best owned by this warp
         const int lane_base = (warp & 3) * 32;        // TMEM lanes this warp may read
-        // Columns are taken 16 at a time.  Column 16*c + j is owned by lane j (c even) or lane
-        // 16 + j (c odd), which keeps that path's running best (key, index) in registers
-        // across all tiles; nothing is exchanged through shared memory until the end.
+        // A group's accumulators finish together.  Columns are then taken 16 at a time and, for
+        // each, the group's tiles are walked with a per-lane running maximum (a lane always sees
+        // increasing vocabulary rows, so a strictly larger value replaces); only then are the
+        // 32 lanes reduced, once per column and group.  Column 16*c + j is owned by lane j
+        // (c even) or lane 16 + j (c odd), which keeps that path's best (key, index) in
+        // registers across groups; nothing goes through shared memory until the end.
         uint32_t best_key[kMaxNPad / 32], best_idx[kMaxNPad / 32];
 #pragma unroll
         for (int c2 = 0; c2 < kMaxNPad / 32; ++c2) { best_key[c2] = 0u; best_idx[c2] = 0u; }
+        const int m = lane_base + lane;
+        const float neg_inf = __uint_as_float(0xFF800000u);
         bool alive = true;
-        for (int tile = 0; tile < my_tiles && alive; ++tile) {
-            const int slot = tile % P.n_slots;
-            // the tcgen05.ld below needs the whole warp: the outcome of the wait is warp-uniform
-            if (!ptx::mbar_wait_warp<kIdlePollNs>(slot_full + 8 * slot, (tile / P.n_slots) & 1, s_abort,
-                                                  kWaitLimitCycles)) {
-                atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_FULL);
-                alive = false;
-                break;
+        for (int g = 0; g < n_groups && alive; ++g) {
+            const int t0 = g * G, t1 = min(my_tiles, t0 + G);
+            for (int tile = t0; tile < t1; ++tile) {
+                // the tcgen05.ld below needs the whole warp: the outcome of the wait is warp-uniform
+                if (!ptx::mbar_wait_warp<kIdlePollNs>(slot_full + 8 * (tile % P.n_slots), (tile / P.n_slots) & 1,
+                                                      s_abort, kWaitLimitCycles)) {
+                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_FULL);
+                    alive = false;
+                    break;
+                }
             }
+            if (!alive) break;
             ptx::tc_fence_after();
-            const int m = lane_base + lane;
-            const int v_tile0 = v_cta0 + tile * P.tile_rows;
-            const int v = v_tile0 + m;
-            const bool valid = (m < P.tile_rows) && (v < P.V);
-            const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(slot * P.n_pad);
 #pragma unroll
             for (int c = 0; c < kMaxNPad / 16; ++c) {
                 const int n0 = c * 16;
                 if (n0 < P.n_pad) {
-                    uint32_t acc[16];
-                    ptx::tmem_ld16(taddr + n0, acc);
-                    ptx::tmem_ld_wait();
-                    if (n0 + 16 >= P.n_pad) {             // accumulator fully read: hand the slot back
+                    float best[16];
+                    int btile[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) { best[j] = neg_inf; btile[j] = t0; }
+                    for (int tile = t0; tile < t1; ++tile) {
+                        const int v = v_cta0 + tile * P.tile_rows + m;
+                        const bool valid = (m < P.tile_rows) && (v < P.V);
+                        uint32_t acc[16];
+                        ptx::tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) +
+                                           (uint32_t)((tile % P.n_slots) * P.n_pad + n0), acc);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float val = __uint_as_float(acc[j]) * P.scale;
+                            if (valid && val > best[j]) { best[j] = val; btile[j] = tile; }
+                        }
+                        if (P.dbg_logits != nullptr && valid) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (n0 + j < P.rows)
+                                    P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
+                                        s_row[n0 + j].q >= 0 ? __uint_as_float(acc[j]) * P.scale
+                                                             : __uint_as_float(0x7FC00000u);
+                        }
+                    }
+                    if (n0 + 16 >= P.n_pad) {   // the group's accumulators are fully read: hand the slots back
                         ptx::tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(slot_empty + 8 * slot);
+                        if (lane == 0)
+                            for (int tile = t0; tile < t1; ++tile) ptx::mbar_arrive(slot_empty + 8 * (tile % P.n_slots));
                     }
-                    uint32_t cur_key = 0u, cur_who = 0u;
+                    uint32_t cur_key = 0u, cur_idx = 0u;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const float val = __uint_as_float(acc[j]) * P.scale;
-                        if (P.dbg_logits != nullptr && valid && n0 + j < P.rows)
-                            P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
-                                s_row[n0 + j].q >= 0 ? val : __uint_as_float(0x7FC00000u);
-                        const uint32_t key = valid ? float_key(val) : 0u;
+                        const uint32_t key = best[j] != neg_inf ? float_key(best[j]) : 0u;
                         const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-                        const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
+                        const uint32_t my_v = (uint32_t)(v_cta0 + btile[j] * P.tile_rows + m);
+                        const uint32_t first = __reduce_min_sync(0xFFFFFFFFu, key == mx ? my_v : 0xFFFFFFFFu);
                         const bool mine = lane == (c & 1) * 16 + j;
                         cur_key = mine ? mx : cur_key;
-                        cur_who = mine ? who : cur_who;
+                        cur_idx = mine ? first : cur_idx;
                     }
-                    // a later tile holds larger indices, so only a strictly larger key replaces
+                    // a later group holds larger indices, so only a strictly larger key replaces
                     if (cur_key > best_key[c >> 1]) {
                         best_key[c >> 1] = cur_key;
-                        best_idx[c >> 1] = (uint32_t)(v_tile0 + lane_base + (__ffs(cur_who) - 1));
+                        best_idx[c >> 1] = cur_idx;
                     }
                 }
             }
