@@ -62,6 +62,7 @@ struct FusedParams {
     int n_slots;      // accumulator slots in TMEM (512 / n_pad)
     int nsw, nsb;     // stages of the W ring and of the operand ring
     int cache_bits;   // keep mask bytes in shared memory after the first group
+    int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
     RowMap map;
     uint32_t key0, key1, thr;
     float scale;
@@ -80,7 +81,8 @@ __device__ __forceinline__ uint32_t mask_pair(uint32_t bits2) {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams P) {
+fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_b,
+                  const FusedParams P) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -104,8 +106,12 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
 
     if (threadIdx.x == 0) {
         ptx::prefetch_tensormap(&tmap_w);
+        if (P.staged) ptx::prefetch_tensormap(&tmap_b);
         for (int s = 0; s < P.nsw; ++s) { ptx::mbar_init(w_full + 8 * s, 1); ptx::mbar_init(w_empty + 8 * s, 1); }
-        for (int s = 0; s < P.nsb; ++s) { ptx::mbar_init(b_ready + 8 * s, wps); ptx::mbar_init(b_empty + 8 * s, 1); }
+        for (int s = 0; s < P.nsb; ++s) {
+            ptx::mbar_init(b_ready + 8 * s, P.staged ? 1 : wps);
+            ptx::mbar_init(b_empty + 8 * s, 1);
+        }
         for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, 4); }
         *s_abort = 0;
         ptx::fence_mbar_init();
@@ -229,13 +235,13 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
         const int lane_base = (warp & 3) * 32;        // TMEM lanes this warp may read
         // A group's accumulators finish together.  Columns are then taken 16 at a time and, for
         // each, the group's tiles are walked with a per-lane running maximum (a lane always sees
-        // increasing vocabulary rows, so a strictly larger value replaces); only then are the
-        // 32 lanes reduced, once per column and group.  Column 16*c + j is owned by lane j
-        // (c even) or lane 16 + j (c odd), which keeps that path's best (key, index) in
-        // registers across groups; nothing goes through shared memory until the end.
-        uint32_t best_key[kMaxNPad / 32], best_idx[kMaxNPad / 32];
-#pragma unroll
-        for (int c2 = 0; c2 < kMaxNPad / 32; ++c2) { best_key[c2] = 0u; best_idx[c2] = 0u; }
+        // increasing vocabulary rows, so a strictly larger value replaces).  Only then are the
+        // 32 lanes reduced, once per column and group, by a halving exchange: in each of four
+        // rounds a lane hands half of its packed (key, inverted index) columns to its partner
+        // and keeps the maxima of the other half, so that 16 columns cost 16 exchanges, not 80.
+        unsigned long long* my_best = s_best + ew * P.n_pad;
+        for (int n = lane; n < P.n_pad; n += 32) my_best[n] = 0ull;
+        __syncwarp();
         const int m = lane_base + lane;
         const float neg_inf = __uint_as_float(0xFF800000u);
         bool alive = true;
@@ -252,67 +258,96 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
             }
             if (!alive) break;
             ptx::tc_fence_after();
+            const int slot0 = t0 % P.n_slots;
+            const int v0 = v_cta0 + t0 * P.tile_rows + m;     // this lane's vocabulary row in tile t0
+#pragma unroll 1
+            for (int n0 = 0; n0 < P.n_pad; n0 += 16) {
+                float best[16];
+                int bv[16];
 #pragma unroll
-            for (int c = 0; c < kMaxNPad / 16; ++c) {
-                const int n0 = c * 16;
-                if (n0 < P.n_pad) {
-                    float best[16];
-                    int btile[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) { best[j] = neg_inf; btile[j] = t0; }
-                    for (int tile = t0; tile < t1; ++tile) {
-                        const int v = v_cta0 + tile * P.tile_rows + m;
-                        const bool valid = (m < P.tile_rows) && (v < P.V);
-                        uint32_t acc[16];
-                        ptx::tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) +
-                                           (uint32_t)((tile % P.n_slots) * P.n_pad + n0), acc);
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float val = __uint_as_float(acc[j]) * P.scale;
-                            if (valid && val > best[j]) { best[j] = val; btile[j] = tile; }
-                        }
-                        if (P.dbg_logits != nullptr && valid) {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (n0 + j < P.rows)
-                                    P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
-                                        s_row[n0 + j].q >= 0 ? __uint_as_float(acc[j]) * P.scale
-                                                             : __uint_as_float(0x7FC00000u);
-                        }
-                    }
-                    if (n0 + 16 >= P.n_pad) {   // the group's accumulators are fully read: hand the slots back
-                        ptx::tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0)
-                            for (int tile = t0; tile < t1; ++tile) ptx::mbar_arrive(slot_empty + 8 * (tile % P.n_slots));
-                    }
-                    uint32_t cur_key = 0u, cur_idx = 0u;
+                for (int j = 0; j < 16; ++j) { best[j] = neg_inf; bv[j] = 0; }
+                int slot = slot0, v = v0;
+                for (int tile = t0; tile < t1; ++tile, v += P.tile_rows) {
+                    const bool valid = (m < P.tile_rows) && (v < P.V);
+                    uint32_t acc[16];
+                    ptx::tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(slot * P.n_pad + n0), acc);
+                    ptx::tmem_ld_wait();
+                    if (++slot == P.n_slots) slot = 0;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const uint32_t key = best[j] != neg_inf ? float_key(best[j]) : 0u;
-                        const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-                        const uint32_t my_v = (uint32_t)(v_cta0 + btile[j] * P.tile_rows + m);
-                        const uint32_t first = __reduce_min_sync(0xFFFFFFFFu, key == mx ? my_v : 0xFFFFFFFFu);
-                        const bool mine = lane == (c & 1) * 16 + j;
-                        cur_key = mine ? mx : cur_key;
-                        cur_idx = mine ? first : cur_idx;
+                        const float val = __uint_as_float(acc[j]) * P.scale;
+                        if (valid && val > best[j]) { best[j] = val; bv[j] = v; }
                     }
-                    // a later group holds larger indices, so only a strictly larger key replaces
-                    if (cur_key > best_key[c >> 1]) {
-                        best_key[c >> 1] = cur_key;
-                        best_idx[c >> 1] = cur_idx;
+                    if (P.dbg_logits != nullptr && valid) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (n0 + j < P.rows)
+                                P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
+                                    s_row[n0 + j].q >= 0 ? __uint_as_float(acc[j]) * P.scale
+                                                         : __uint_as_float(0x7FC00000u);
                     }
+                }
+                if (n0 + 16 >= P.n_pad) {   // the group's accumulators are fully read: hand the slots back
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        int sl = slot0;
+                        for (int tile = t0; tile < t1; ++tile) {
+                            ptx::mbar_arrive(slot_empty + 8 * sl);
+                            if (++sl == P.n_slots) sl = 0;
+                        }
+                    }
+                }
+                unsigned long long p16[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    p16[j] = best[j] != neg_inf ? pack_best(float_key(best[j]), (uint32_t)bv[j]) : 0ull;
+                unsigned long long p8[8], p4[4], p2[2], p1;
+                {
+                    const bool up = (lane & 16) != 0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const unsigned long long give = up ? p16[j] : p16[j + 8], keep = up ? p16[j + 8] : p16[j];
+                        const unsigned long long got = __shfl_xor_sync(0xFFFFFFFFu, give, 16);
+                        p8[j] = got > keep ? got : keep;
+                    }
+                }
+                {
+                    const bool up = (lane & 8) != 0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned long long give = up ? p8[j] : p8[j + 4], keep = up ? p8[j + 4] : p8[j];
+                        const unsigned long long got = __shfl_xor_sync(0xFFFFFFFFu, give, 8);
+                        p4[j] = got > keep ? got : keep;
+                    }
+                }
+                {
+                    const bool up = (lane & 4) != 0;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const unsigned long long give = up ? p4[j] : p4[j + 2], keep = up ? p4[j + 2] : p4[j];
+                        const unsigned long long got = __shfl_xor_sync(0xFFFFFFFFu, give, 4);
+                        p2[j] = got > keep ? got : keep;
+                    }
+                }
+                {
+                    const bool up = (lane & 2) != 0;
+                    const unsigned long long give = up ? p2[0] : p2[1], keep = up ? p2[1] : p2[0];
+                    const unsigned long long got = __shfl_xor_sync(0xFFFFFFFFu, give, 2);
+                    p1 = got > keep ? got : keep;
+                }
+                {
+                    const unsigned long long got = __shfl_xor_sync(0xFFFFFFFFu, p1, 1);
+                    p1 = got > p1 ? got : p1;
+                }
+                // lanes 2x and 2x+1 now hold column 8*bit4 + 4*bit3 + 2*bit2 + bit1 of the chunk
+                if ((lane & 1) == 0) {
+                    const int n = n0 + (lane >> 1);
+                    if (p1 > my_best[n]) my_best[n] = p1;   // equal keys: the smaller index packs larger
                 }
             }
         }
-        unsigned long long* my_best = s_best + ew * P.n_pad;
-#pragma unroll
-        for (int c = 0; c < kMaxNPad / 16; ++c) {
-            const int n = c * 16 + (lane & 15);
-            if (n < P.n_pad && (lane >> 4) == (c & 1))
-                my_best[n] = best_key[c >> 1] != 0u ? pack_best(best_key[c >> 1], best_idx[c >> 1]) : 0ull;
-        }
+        __syncwarp();
         ptx::bar_sync(1, 4 * 32);
         for (int n = threadIdx.x - kFirstEpiWarp * 32; n < P.rows; n += 4 * 32) {
             unsigned long long b = s_best[n];
@@ -335,6 +370,27 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
             ptx::tmem_dealloc(tmem_base, kTmemCols);
         }
     } else {
+        if (P.staged) {
+            // -------------------------------------------------------------- operand producer
+            // The masked rows were written to the staging buffer by mask_operand_kernel; one
+            // thread streams the [n_pad x 64] block of every (group, block) step through TMA.
+            if (threadIdx.x != kFirstExpWarp * 32) return;
+            const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+            uint32_t bar_r = b_ready, bar_e = b_empty, dst = smem_base + P.off_b, parity = 1;
+            int stage = 0;
+            for (int g = 0; g < n_groups; ++g)
+                for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_e, parity, s_abort, kWaitLimitCycles)) {
+                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                        return;
+                    }
+                    ptx::mbar_arrive_expect_tx(bar_r, b_stage_bytes);
+                    ptx::tma_load_2d(dst, &tmap_b, x, P.row0, bar_r);
+                    bar_r += 8; bar_e += 8; dst += b_stage_bytes;
+                    if (++stage == P.nsb) { stage = 0; parity ^= 1; bar_r = b_ready; bar_e = b_empty; dst = smem_base + P.off_b; }
+                }
+            return;
+        }
         // ------------------------------------------------------------------ operand builders
         const int e = warp - kFirstExpWarp;
         const int grp = e % P.nsb, sub = e / P.nsb;
@@ -421,6 +477,29 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
 
 }
 
+// Eq. 1 and the numerator of Eq. 2 for every path of a call whose rows do not fit the
+// in-kernel builders: row r of the staging buffer receives hidden row q(r) with the dropped
+// elements zeroed.  One thread per 16-byte chunk (two Philox quads).
+__global__ void __launch_bounds__(256)
+mask_operand_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat16* __restrict__ out, int rows, int d,
+                    RowMap map, uint32_t key0, uint32_t key1, uint32_t thr, uint32_t* __restrict__ err) {
+    const int chunks = d >> 3;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)rows * chunks) return;
+    const int r = (int)(idx / chunks), c = (int)(idx - (long long)r * chunks);
+    RowKey k;
+    if (!row_key(map, r, k) && c == 0) atomicExch(err, (uint32_t)ERR_BAD_ROW);
+    const uint32_t mbits = keep4((uint32_t)(2 * c), k, key0, key1, thr) |
+                           (keep4((uint32_t)(2 * c + 1), k, key0, key1, thr) << 4);
+    const uint4 hv = __ldg(reinterpret_cast<const uint4*>(H + (size_t)k.q * d + c * 8));
+    uint4 o;
+    o.x = hv.x & mask_pair(mbits);
+    o.y = hv.y & mask_pair(mbits >> 2);
+    o.z = hv.z & mask_pair(mbits >> 4);
+    o.w = hv.w & mask_pair(mbits >> 6);
+    *reinterpret_cast<uint4*>(out + (size_t)r * d + c * 8) = o;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------ host side
@@ -428,6 +507,11 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const FusedParams 
 struct FusedState {
     CUtensorMap tmap_w;
     int n_ctas, tiles_per_cta, tile_rows, slice_rows;
+    // staging buffer for the masked operand of calls with too many rows for the in-kernel
+    // builders, and one tensor map per box height n_pad = 16, 32, ..., 256 over it
+    __nv_bfloat16* staging;
+    int staging_rows;
+    CUtensorMap tmap_b[kMaxNPad / 16];
 };
 
 namespace {
@@ -451,50 +535,55 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 struct SmemPlan {
-    int nsw, nsb, cache_bits, group_tiles, n_slots;
+    int nsw, nsb, cache_bits, group_tiles, n_slots, staged;
     uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar, total;
 };
 
 // Choose the tile grouping, then split the 227 KB of shared memory between the W ring, the
 // operand ring and (only when tiles need more than one group) the mask cache.
 bool plan_smem(int rows, int n_pad, int d, int tiles_per_cta, SmemPlan* out) {
+    (void)rows; (void)d;
     SmemPlan best{};
     best.n_slots = kTmemCols / n_pad;
-    if (tiles_per_cta <= best.n_slots) {
-        best.group_tiles = tiles_per_cta;               // the whole slice is live at once
-    } else {
-        // several groups: use half of the slots per group so that the epilogue of one group
-        // overlaps the MMAs of the next, and even the group sizes out
-        int g = best.n_slots / 2 > 0 ? best.n_slots / 2 : 1;
-        const int n_groups = (tiles_per_cta + g - 1) / g;
-        best.group_tiles = (tiles_per_cta + n_groups - 1) / n_groups;
-    }
-    const bool multi = best.group_tiles < tiles_per_cta;
-    const int kb_count = d / kBlockK;
     const uint32_t b_stage = (uint32_t)n_pad * (kBlockK * 2);
-    const uint32_t bits = ((uint32_t)rows * (uint32_t)(d / 8) + 15u) & ~15u;
     const uint32_t fixed = 256u * sizeof(RowInfo) + 4u * n_pad * 8u + kBarBytes;
     const uint32_t avail = kSmemLimit - 1024 - fixed;
-    int best_score = -1;
-    for (int cache = multi ? 1 : 0; cache >= 0; --cache)
-        for (int nsb = 4; nsb >= 2; nsb >>= 1) {
-            if (cache && (kb_count % nsb) != 0) continue;
-            const uint64_t used = (uint64_t)nsb * b_stage + (cache ? bits : 0u);
-            if (used + 2u * kWStageBytes > avail) continue;
-            int nsw = (int)((avail - used) / kWStageBytes);
-            if (nsw > kMaxWStages) nsw = kMaxWStages;
-            // prefer: at least six W stages, then the mask cache, then deeper rings
-            const int score = (nsw >= 6 ? 1000 : 0) + cache * 100 + nsb * 4 + nsw;
-            if (score > best_score) {
-                best_score = score;
-                best.nsw = nsw; best.nsb = nsb; best.cache_bits = cache;
-            }
+    if (tiles_per_cta <= best.n_slots) {
+        // One group: the whole slice is live at once and the builders generate the masks in
+        // registers, once per call.  Four small operand stages, the rest goes to the W ring.
+        best.group_tiles = tiles_per_cta;
+        best.staged = 0;
+        best.nsb = 4;
+    } else {
+        // Several groups: the operand would have to be rebuilt for every group, so it is staged
+        // through global memory by mask_operand_kernel and streamed in by TMA (no builders).
+        // With four or more slots a group takes half of them, so that the epilogue of one group
+        // overlaps the MMAs of the next; with fewer, a group takes them all, which halves the
+        // operand traffic and leaves the epilogue exposed.  Group sizes are evened out.
+        int g = best.n_slots >= 4 ? best.n_slots / 2 : best.n_slots;
+        const int n_groups = (tiles_per_cta + g - 1) / g;
+        best.group_tiles = (tiles_per_cta + n_groups - 1) / n_groups;
+        best.staged = 1;
+        // operand ring: up to 96 KB, two to four stages (a stage lasts group_tiles W steps)
+        best.nsb = (int)(96u * 1024u / b_stage);
+        if (best.nsb > 4) best.nsb = 4;
+        if (best.nsb < 2) best.nsb = 2;
+    }
+    best.cache_bits = 0;
+    for (;;) {   // shrink the operand ring until the W ring has six stages (or the ring is at two)
+        const uint32_t used = (uint32_t)best.nsb * b_stage;
+        if (used + 2u * kWStageBytes <= avail) {
+            best.nsw = (int)((avail - used) / kWStageBytes);
+            if (best.nsw > kMaxWStages) best.nsw = kMaxWStages;
+            if (best.nsw >= 6 || best.nsb == 2) break;
         }
-    if (best_score < 0) return false;
+        if (best.nsb == 2) return false;
+        best.nsb = best.staged ? best.nsb - 1 : 2;   // the eight builder warps split evenly over 4 or 2 stages
+    }
     best.off_w = 0;
     best.off_b = (uint32_t)best.nsw * kWStageBytes;
     best.off_bits = best.off_b + (uint32_t)best.nsb * b_stage;
-    best.off_rowinfo = best.off_bits + (best.cache_bits ? bits : 0u);
+    best.off_rowinfo = best.off_bits;
     best.off_best = best.off_rowinfo + 256u * sizeof(RowInfo);
     best.off_bar = best.off_best + 4u * n_pad * 8u;
     best.total = best.off_bar + kBarBytes + 1024u;
@@ -508,7 +597,7 @@ bool fused_supported(const HeadDesc& head, int rows) {
     return head.dtype == DM_BF16 && head.d >= kBlockK && head.d % kBlockK == 0 && head.V >= 1 && rows >= 1;
 }
 
-int fused_create(FusedState** out, const HeadDesc& head, int /*max_rows*/, int /*max_hidden_rows*/,
+int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max_hidden_rows*/,
                  size_t* bytes) {
     *out = nullptr;
     *bytes = 0;
@@ -542,17 +631,44 @@ int fused_create(FusedState** out, const HeadDesc& head, int /*max_rows*/, int /
         delete fs;
         return DM_ECUDA;
     }
+    // Staging buffer, only if the largest launch this context may see needs it.
+    fs->staging = nullptr;
+    fs->staging_rows = 0;
+    const int widest = max_rows < kMaxNPad ? max_rows : kMaxNPad;
+    SmemPlan plan;
+    if (!plan_smem(widest, (widest + 15) & ~15, head.d, fs->tiles_per_cta, &plan)) { delete fs; return DM_EUNSUPPORTED; }
+    if (plan.staged) {
+        fs->staging_rows = (max_rows + 15) & ~15;
+        const size_t n = (size_t)fs->staging_rows * head.d * sizeof(__nv_bfloat16);
+        if (cudaMalloc(&fs->staging, n) != cudaSuccess) { cudaGetLastError(); delete fs; return DM_ECUDA; }
+        if (cudaMemset(fs->staging, 0, n) != cudaSuccess) { cudaGetLastError(); cudaFree(fs->staging); delete fs; return DM_ECUDA; }
+        const cuuint64_t sdim[2] = {(cuuint64_t)head.d, (cuuint64_t)fs->staging_rows};
+        for (int n16 = 1; n16 <= kMaxNPad / 16; ++n16) {
+            const cuuint32_t sbox[2] = {(cuuint32_t)kBlockK, (cuuint32_t)(16 * n16)};
+            if (16 * n16 > fs->staging_rows) { fs->tmap_b[n16 - 1] = fs->tmap_b[0]; continue; }
+            r = encode(&fs->tmap_b[n16 - 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, fs->staging, sdim, gstride, sbox,
+                       estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) { cudaFree(fs->staging); delete fs; return DM_ECUDA; }
+        }
+        *bytes = n;
+    }
     *out = fs;
     return DM_OK;
 }
 
-void fused_destroy(FusedState* fs) { delete fs; }
+void fused_destroy(FusedState* fs) {
+    if (fs == nullptr) return;
+    cudaFree(fs->staging);
+    delete fs;
+}
 
 int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hidden*/, int rows,
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out) {
     if (fs == nullptr || !fused_supported(head, rows) || fs->n_ctas > kMaxSlices) return DM_EUNSUPPORTED;
     int launches = 0;
+    bool operand_staged = false;
     for (int row0 = 0; row0 < rows; row0 += kMaxNPad) {
         FusedParams P{};
         P.H = static_cast<const __nv_bfloat16*>(H);
@@ -565,13 +681,24 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         SmemPlan plan;
         if (!plan_smem(P.rows, P.n_pad, head.d, fs->tiles_per_cta, &plan)) return DM_EUNSUPPORTED;
         P.group_tiles = plan.group_tiles; P.n_slots = plan.n_slots;
-        P.nsw = plan.nsw; P.nsb = plan.nsb; P.cache_bits = plan.cache_bits;
+        P.nsw = plan.nsw; P.nsb = plan.nsb; P.cache_bits = plan.cache_bits; P.staged = plan.staged;
+        if (plan.staged && !operand_staged) {
+            // one pass over all rows of the call; the launches below read their own rows of it
+            if (fs->staging == nullptr || rows > fs->staging_rows) return DM_EWORKSPACE;
+            const long long n_threads = (long long)rows * (head.d / 8);
+            mask_operand_kernel<<<(unsigned)((n_threads + 255) / 256), 256, 0, stream>>>(
+                static_cast<const __nv_bfloat16*>(H), fs->staging, rows, head.d, map, mk.key0, mk.key1, mk.thr, err);
+            if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
+            operand_staged = true;
+            ++launches;
+        }
         P.off_w = plan.off_w; P.off_b = plan.off_b; P.off_bits = plan.off_bits;
         P.off_rowinfo = plan.off_rowinfo; P.off_best = plan.off_best; P.off_bar = plan.off_bar;
         P.map = map;
         P.key0 = mk.key0; P.key1 = mk.key1; P.thr = mk.thr; P.scale = mk.scale;
         P.partials = partials; P.dbg_logits = dbg_logits; P.err = err;
-        fused_head_kernel<<<fs->n_ctas, kThreads, plan.total, stream>>>(fs->tmap_w, P);
+        fused_head_kernel<<<fs->n_ctas, kThreads, plan.total, stream>>>(
+            fs->tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : fs->tmap_w, P);
         if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
         ++launches;
     }
