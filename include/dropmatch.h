@@ -53,7 +53,8 @@ enum {
     DM_ECUDA = -3,        /* a CUDA runtime or driver call failed                               */
     DM_EWORKSPACE = -4,   /* call needs more rows than dm_set_head reserved                     */
     DM_EDEVICE = -5,      /* device is not compute capability 10.x                              */
-    DM_ENOHEAD = -6       /* dm_set_head has not been called                                    */
+    DM_ENOHEAD = -6,      /* dm_set_head has not been called                                    */
+    DM_ESTATICLIMIT = -7  /* call exceeds DM_STATIC_MAX_ROWS of dropmatch_verify_batched_static */
 };
 enum { DM_F32 = 0, DM_BF16 = 1 };             /* storage type of W and H (accumulation is fp32) */
 enum { DM_RULE_NAIVE = 0, DM_RULE_MAJORITY = 1 };
@@ -107,6 +108,33 @@ int dropmatch_verify_batched_host(dm_ctx* ctx, const void* H_host, const int32_t
                                   int32_t* out_tokens_host, int32_t* out_counts_host,
                                   int32_t* out_draft_hits_host, int32_t* out_accept_len_host,
                                   void* stream);
+
+/* The paper has no counterpart to this entry point; it exists for the way the library gets
+ * deployed.  Some hosts of this code cannot ask CUDA for device memory at the time they verify:
+ * a serving process that hands all of HBM to its own pool at start-up (a later cudaMalloc fails
+ * or eats into the KV cache), a latency-critical decode loop (cudaMalloc and cudaFree stall the
+ * whole device), or a plug-in that is handed tensors but may not set up a context with a
+ * workspace of its own.  For them this call does what dropmatch_verify_batched does on the
+ * CUDA-core kernel family, for fp32 and bf16 heads alike, but needs no dm_ctx and never
+ * allocates or frees: the per-slice partial argmaxes go to a fixed array inside the library
+ * image (about 0.6 MB, held by every GPU that loads the library until the process exits).
+ *   device           CUDA device of all the pointers (compute capability 10.x)
+ *   W[V,d], dtype    the LM head, as for dm_set_head (device pointer, 16-byte aligned)
+ *   the rest         as for dropmatch_verify_batched; out_draft_hits may be NULL
+ * Limits and rules:
+ *   - B*T*K <= DM_STATIC_MAX_ROWS, else DM_ESTATICLIMIT and nothing is launched.
+ *   - The first call on a device looks the array's device address up (once per device and
+ *     process).  Make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     call itself clears the part that must start at zero.  Two calls whose kernels can overlap
+ *     on the GPU (different streams, or host threads racing on one device) corrupt each other:
+ *     issue them on one stream, or order them with events.
+ *   - Only enqueues work on `stream`; results are ready when the stream reaches that point. */
+#define DM_STATIC_MAX_ROWS 256
+int dropmatch_verify_batched_static(int device, const void* W, int V, int d, int dtype, const void* H,
+                                    const int32_t* draft, int B, int T, int K, float p, uint64_t seed,
+                                    uint64_t seq_base, int rule, int32_t* out_tokens, int32_t* out_counts,
+                                    int32_t* out_draft_hits, int32_t* out_accept_len, void* stream);
 
 /* Draft trees (Sec. 4.4).  Per sequence: N_h hidden rows H[b,q,:] and N nodes in topological
  * order.  Node n has a token, a parent node (node_parent[n] < n; -1 = child of the committed

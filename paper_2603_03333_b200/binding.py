@@ -11,7 +11,8 @@ from pathlib import Path
 
 import torch
 
-OK, EINVAL, EUNSUPPORTED, ECUDA, EWORKSPACE, EDEVICE, ENOHEAD = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, EUNSUPPORTED, ECUDA, EWORKSPACE, EDEVICE, ENOHEAD, ESTATICLIMIT = 0, -1, -2, -3, -4, -5, -6, -7
+STATIC_MAX_ROWS = 256
 F32, BF16 = 0, 1
 RULE_NAIVE, RULE_MAJORITY = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
@@ -30,6 +31,8 @@ SIGNATURES = {
     "dropmatch_verify": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _u64, _ci, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_batched_static": (_ci, [_ci, _vp, _ci, _ci, _ci, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
+                                              _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_tree": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
                                     _vp, _vp, _vp, _vp, _vp, _vp]),
     "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
@@ -85,6 +88,27 @@ def _dev(t: torch.Tensor, dtype, what: str) -> torch.Tensor:
     if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
         raise TypeError(f"{what} must be a contiguous CUDA tensor of {dtype}")
     return t
+
+
+def verify_batched_static(W, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE, out=None):
+    """dropmatch_verify_batched_static: chain verification without a context and without any
+    device allocation inside the library (the output tensors are the caller's; pass `out` to
+    reuse them).  B*T*K may not exceed STATIC_MAX_ROWS."""
+    if W.dtype not in (torch.float32, torch.bfloat16) or not W.is_cuda or not W.is_contiguous() or W.dim() != 2:
+        raise TypeError("W must be a contiguous 2-D CUDA tensor of float32 or bfloat16")
+    dtype = F32 if W.dtype == torch.float32 else BF16
+    _dev(H, W.dtype, "H"); _dev(draft, torch.int32, "draft")
+    B, T, _ = H.shape
+    V, d = W.shape
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=W.device)
+        out = dict(tokens=torch.empty((B, T, K), **i32), counts=torch.empty((B, T, K), **i32),
+                   hits=torch.empty((B, T), **i32), accept_len=torch.empty((B,), **i32))
+    _check(lib().dropmatch_verify_batched_static(W.device.index, _ptr(W), V, d, dtype, _ptr(H), _ptr(draft), B, T, K,
+                                                 p, seed, seq_base, rule, _ptr(out["tokens"]), _ptr(out["counts"]),
+                                                 _ptr(out["hits"]), _ptr(out["accept_len"]), _stream(W.device)),
+           "dropmatch_verify_batched_static")
+    return out
 
 
 class Context:

@@ -397,6 +397,7 @@ const char* dm_strerror(int status) {
         case DM_EWORKSPACE: return "call exceeds the rows reserved by dm_set_head";
         case DM_EDEVICE: return "device is not compute capability 10.x";
         case DM_ENOHEAD: return "dm_set_head has not been called";
+        case DM_ESTATICLIMIT: return "call exceeds the fixed scratch of dropmatch_verify_batched_static";
         default: return "unknown status";
     }
 }
