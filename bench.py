@@ -111,6 +111,24 @@ def time_oracle(cfg, work_cpu, steps, warmup, budget_s=20.0):
     return 1.0 / t_call, oracle.threads(), sample, t_call * 1e3
 
 
+def max_over_ranks(x: float, world: int, device="cpu") -> float:
+    """The slowest rank's figure (replicas run independently; the job is as slow as its slowest)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_calls_per_s(ms_total_local: float, steps: int, world: int, device="cpu"):
+    """Whole-job throughput of `world` independent replicas that each ran `steps` verify calls:
+    (world * steps) / (max over ranks of the timed region).  Returns (calls/s, ms per step)."""
+    ms_total = max_over_ranks(ms_total_local, world, device)
+    return world * steps / (ms_total * 1e-3), ms_total / steps
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -182,12 +200,7 @@ def run_cuda(args):
     ms_total = ev0.elapsed_time(ev1)
     launches_per_step = ctx.last_launches()
     impl_used = ctx.last_impl()
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    ms_step = ms_total / args.steps
-    value = world * args.steps / (ms_total * 1e-3)
+    value, ms_step = aggregate_calls_per_s(ms_total, args.steps, world, dev)
 
     # dominant kernel alone: events on the launching stream around the head kernel of each step
     ctx.profile_head(True)
@@ -220,10 +233,7 @@ def run_cuda(args):
         ctx.verify_batched_host(Hh, dh, cfg.K, cfg.p, seed + i, out=hout)   # returns after the D2H copy
     torch.cuda.synchronize()
     e_s = time.perf_counter() - e0
-    te = torch.tensor([e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e = dict(value=world * n_e2e / float(te.item()), unit=UNIT,
+    e2e = dict(value=aggregate_calls_per_s(e_s * 1e3, n_e2e, world, dev)[0], unit=UNIT,
                h2d_bytes_per_step=Hh.numel() * elem + dh.numel() * 4,
                d2h_bytes_per_step=sum(v.numel() * 4 for v in hout.values()))
 
@@ -250,7 +260,7 @@ def run_cuda(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=WORKLOAD)

@@ -1,0 +1,119 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle needs V*d fp64 multiply-adds per path (half a second at the Llama-3-8B head), so it is
+run on a sample of paths: their decoded tokens (outside near-ties) and their full logit rows are
+compared one by one.  Everything that is integer work is checked in full from the GPU's own
+tokens with the oracle's integer routines: multiplicities, hits, accepted lengths, tree walks;
+masks are compared bit for bit on sampled paths."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_03333_b200 as pk
+from paper_2603_03333_b200 import binding, workloads as wl
+from parity_util import NEAR_TIE, TOL_LOGIT_BF16, to_np
+
+pytestmark = pytest.mark.gpu
+SEED = wl.MASK_SEED
+DEV = "cuda:0"
+
+
+def _sample_paths(cfg, n, rng):
+    all_paths = [(b, t, i) for b in range(cfg.B) for t in range(cfg.T) for i in range(cfg.K)]
+    idx = rng.choice(len(all_paths), size=min(n, len(all_paths)), replace=False)
+    return [all_paths[j] for j in sorted(idx)]
+
+
+def _check_sampled_paths(ctx, cfg, work, got_tokens, paths, seq_base=0):
+    Wn, Hn = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H)
+    sel = torch.tensor(paths, dtype=torch.int32, device=DEV)
+    logits = ctx.debug_logits(work.H, sel, cfg.p, SEED, seq_base=seq_base).cpu().numpy()
+    assert ctx.device_error() == 0
+    near = 0
+    for n, (b, t, i) in enumerate(paths):
+        exp = oracle.logits_row(Wn, cfg.dtype, Hn[b, t], cfg.p, SEED, seq_base + b, t, i)
+        assert np.abs(logits[n] - exp).max() < TOL_LOGIT_BF16, (b, t, i)
+        tok, gap = oracle.argmax(exp)
+        if got_tokens[b, t, i] != tok:
+            assert gap < NEAR_TIE, f"path {(b, t, i)}: token {got_tokens[b, t, i]} vs {tok}, gap {gap}"
+            near += 1
+    return near
+
+
+def _check_masks(ctx, cfg, paths, seq_base=0):
+    got = ctx.debug_masks(cfg.B, cfg.T, cfg.K, cfg.d, cfg.p, SEED, seq_base=seq_base).cpu().numpy().view(np.uint32)
+    thr = oracle.drop_threshold(cfg.p)
+    for (b, t, i) in paths[:4]:
+        bits = np.array([oracle.mask_keep(SEED, seq_base + b, t, i, j, thr) for j in range(0, cfg.d, 7)], dtype=np.uint32)
+        js = np.arange(0, cfg.d, 7)
+        assert np.array_equal((got[b, t, i, js // 32] >> (js % 32)) & 1, bits)
+
+
+@pytest.mark.parametrize("name,overrides,n_paths", [
+    ("llama8b", {}, 8),                               # the bench workload: one accumulator group, in-kernel masks
+    ("qwen8b", dict(K=16), 5),                        # 112 rows: staged operand, three groups
+    ("qwen8b", dict(K=32, p=0.2), 4),                 # 224 rows: two accumulator slots, exposed epilogue
+])
+def test_chain_configs_at_full_size(name, overrides, n_paths):
+    cfg = wl.CONFIGS[name].with_(**overrides)
+    work = wl.make_workload(cfg, device=DEV)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+        got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
+        assert ctx.device_error() == 0 and ctx.last_impl() == binding.IMPL_TCGEN05
+        draft = work.draft.cpu().numpy()
+        for b in range(cfg.B):                        # integer stages, in full, from the GPU's tokens
+            for t in range(cfg.T):
+                cnt, hits = oracle.counts(got["tokens"][b, t], int(draft[b, t]))
+                assert np.array_equal(got["counts"][b, t], cnt) and got["hits"][b, t] == hits
+            assert got["accept_len"][b] == oracle.accept_chain(got["tokens"][b], draft[b], oracle.RULE_NAIVE)
+        assert (got["tokens"] >= 0).all() and (got["tokens"] < cfg.V).all()
+        paths = _sample_paths(cfg, n_paths, np.random.default_rng(11))
+        _check_masks(ctx, cfg, paths)
+        _check_sampled_paths(ctx, cfg, work, got["tokens"], paths)
+        # the accepted drafts of this recipe are plausible ones: something is accepted somewhere
+        assert got["hits"].sum() > 0
+    finally:
+        ctx.close()
+
+
+def test_tree_config_at_full_size():
+    cfg0 = wl.CONFIGS["tree"]
+    work = wl.make_workload(cfg0, device=DEV)
+    cfg = work.cfg                                    # T = hidden rows per sequence of the drawn trees
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+        got = to_np(ctx.verify_tree(work.H, work.node_token, work.node_parent, work.node_hrow, cfg.K, cfg.p, SEED))
+        assert ctx.device_error() == 0 and ctx.last_impl() == binding.IMPL_TCGEN05
+        nt, npar, nh = (x.cpu().numpy() for x in (work.node_token, work.node_parent, work.node_hrow))
+        for b in range(cfg.B):
+            L, best, ok = oracle.accept_tree(got["tokens"][b], nt[b], npar[b], nh[b], oracle.RULE_NAIVE)
+            assert got["accept_len"][b] == L and got["best_node"][b] == best
+            assert np.array_equal(got["node_ok"][b], ok)
+            assert 0 <= L <= 7
+            for q in range(cfg.T):
+                assert np.array_equal(got["counts"][b, q], oracle.counts(got["tokens"][b, q], -1)[0])
+        paths = _sample_paths(cfg, 4, np.random.default_rng(12))
+        _check_sampled_paths(ctx, cfg, work, got["tokens"], paths)
+    finally:
+        ctx.close()
+
+
+def test_llama70b_config_sampled():
+    cfg = wl.CONFIGS["llama70b"]
+    work = wl.make_workload(cfg, device=DEV)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+        got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
+        assert ctx.device_error() == 0
+        draft = work.draft.cpu().numpy()
+        for b in range(cfg.B):
+            assert got["accept_len"][b] == oracle.accept_chain(got["tokens"][b], draft[b], oracle.RULE_NAIVE)
+        paths = _sample_paths(cfg, 3, np.random.default_rng(13))
+        _check_sampled_paths(ctx, cfg, work, got["tokens"], paths)
+    finally:
+        ctx.close()
