@@ -97,9 +97,11 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
         ev_end = c->prof_events[c->prof_used + 1];
         cudaEventRecord(ev_begin, stream);
     }
+    bool folded = false;
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
-                          nullptr, c->err, stream, &launches);
+                          nullptr, c->err, stream, &launches, &fa, c->err + 1,
+                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded);
     else {
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, stream);
         launches = 1;
@@ -109,10 +111,13 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
         c->prof_used += 2;
     }
     if (st != DM_OK) return st;
-    st = launch_finalize(c->partials, n_slices, rows, fa, stream);
-    if (st != DM_OK) return st;
+    if (!folded) {   // calls of several launches, and the CUDA-core family, finish in a kernel of their own
+        st = launch_finalize(c->partials, n_slices, rows, fa, stream);
+        if (st != DM_OK) return st;
+        ++launches;
+    }
     c->last_impl = impl;
-    c->last_launches = launches + 1;
+    c->last_launches = launches;
     return DM_OK;
 }
 
@@ -143,8 +148,9 @@ int dm_create(dm_ctx** out, int device) {
     dm_ctx* c = new (std::nothrow) dm_ctx();
     if (c == nullptr) return DM_ECUDA;
     c->device = device;
-    if (cudaMalloc(&c->err, sizeof(uint32_t)) != cudaSuccess ||
-        cudaMemset(c->err, 0, sizeof(uint32_t)) != cudaSuccess) {
+    // two words: the device error word, then the finished-CTA ticket of the fused kernel
+    if (cudaMalloc(&c->err, 2 * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(c->err, 0, 2 * sizeof(uint32_t)) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(c->err);
         delete c;
@@ -180,11 +186,15 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
     free_workspace(c);
     c->has_head = false;
     const size_t elem = dtype == DM_F32 ? 4 : 2;
-    const size_t n_part = (size_t)kMaxSlices * max_rows * sizeof(unsigned long long);
+    // per-slice partial argmaxes [kMaxSlices][max_rows], then the per-row running best [max_rows]
+    // that the fused kernel's CTAs reduce into when one launch covers the call (zero between calls)
+    const size_t n_part = ((size_t)kMaxSlices + 1) * max_rows * sizeof(unsigned long long);
     const size_t n_H = (size_t)max_hidden_rows * d * elem;
     const size_t n_i32 = ((size_t)3 * max_hidden_rows + 2 * (size_t)max_rows) * sizeof(int32_t);
     if (cudaMalloc(&c->partials, n_part) != cudaSuccess || cudaMalloc(&c->stage_H, n_H) != cudaSuccess ||
-        cudaMalloc(&c->stage_i32, n_i32) != cudaSuccess) {
+        cudaMalloc(&c->stage_i32, n_i32) != cudaSuccess ||
+        cudaMemset(c->partials + (size_t)kMaxSlices * max_rows, 0, (size_t)max_rows * sizeof(unsigned long long)) !=
+            cudaSuccess) {
         cudaGetLastError();
         free_workspace(c);
         return DM_ECUDA;
@@ -347,9 +357,17 @@ int dm_device_error(dm_ctx* c, void* stream, uint32_t* out_code) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint32_t code = 0;
     if (cudaMemcpyAsync(&code, c->err, sizeof code, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemsetAsync(c->err, 0, sizeof code, s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaMemsetAsync(c->err, 0, 2 * sizeof code, s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) {
         cudaGetLastError();
         return DM_ECUDA;
+    }
+    if (code != 0 && c->partials != nullptr) {   // a call that gave up may have left partial maxima behind
+        if (cudaMemsetAsync(c->partials + (size_t)kMaxSlices * c->max_rows, 0,
+                            (size_t)c->max_rows * sizeof(unsigned long long), s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            cudaGetLastError();
+            return DM_ECUDA;
+        }
     }
     *out_code = code;
     return DM_OK;

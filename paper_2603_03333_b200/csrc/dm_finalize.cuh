@@ -1,0 +1,144 @@
+// Split-V merge, token histogram and acceptance of one sequence (Sec. 3.2: naive token matching,
+// Eq. 6 majority; left-to-right rule; tree drafts of Sec. 4.4), as a device routine that a group
+// of threads runs together: the finalize kernel (one block per sequence) and the last CTA of
+// the fused head kernel (its four epilogue warps, sequence after sequence) both call it.
+#pragma once
+#include "dm_internal.h"
+
+namespace dm {
+
+struct BlockSync {
+    __device__ __forceinline__ void operator()() const { __syncthreads(); }
+};
+// bar.sync on a named barrier among `threads` threads (a multiple of 32, whole warps).
+struct NamedSync {
+    int id, threads;
+    __device__ __forceinline__ void operator()() const {
+        asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+    }
+};
+
+// Does `draft` pass `rule` against the K tokens of one hidden row (shared memory)?
+__device__ __forceinline__ bool position_ok(const int32_t* toks, int K, int32_t draft, int rule,
+                                            int* hits_out) {
+    int hits = 0;
+    for (int i = 0; i < K; ++i) hits += (toks[i] == draft);
+    if (hits_out) *hits_out = hits;
+    if (rule == DM_RULE_NAIVE) return hits >= 1;
+    // Eq. 6: draft must be the most frequent token; equal frequencies -> smallest id wins.
+    if (hits == 0) return false;
+    for (int i = 0; i < K; ++i) {
+        int32_t y = toks[i];
+        if (y == draft) continue;
+        int c = 0;
+        for (int i2 = 0; i2 < K; ++i2) c += (toks[i2] == y);
+        if (c > hits || (c == hits && y < draft)) return false;
+    }
+    return true;
+}
+
+// Sequence b of a call of `rows` paths whose per-slice partial argmaxes are partials[slice][row].
+// `sm` is scratch shared memory of finalize_smem_bytes(T, K, N) bytes; thread `tid` of `nthreads`.
+template <class Sync>
+__device__ __forceinline__ void finalize_sequence(const unsigned long long* partials, int n_slices, int rows,
+                                                  const FinalizeArgs& a, int b, int32_t* sm, int tid,
+                                                  int nthreads, Sync sync) {
+    const int TK = a.T * a.K;
+    int32_t* toks = sm;            // [T*K]
+    int32_t* flag = sm + TK;       // chain: ok[T]; tree: test[N] then ok/depth packed [N]
+    const size_t row0 = (size_t)b * TK;
+
+    // split-V merge: the packed (key, inverted index) maximum over slices is the argmax with
+    // the smallest index on ties.  Many slices: one warp per row, lanes stride over the slices.
+    // Few slices (the fused kernel's CTAs have already reduced into one): one thread per row, so
+    // that all loads of a sequence are in flight together.
+    const int warp = tid >> 5, lane = tid & 31, n_warps = nthreads >> 5;
+    if (n_slices < 32) {
+        for (int x = tid; x < TK; x += nthreads) {
+            unsigned long long best = 0ull;
+            for (int s = 0; s < n_slices; ++s) {
+                unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x);
+                best = c > best ? c : best;
+            }
+            int32_t tok = (int32_t)best_index(best);
+            toks[x] = tok;
+            a.out_tokens[row0 + x] = tok;
+        }
+    } else {
+        for (int x = warp; x < TK; x += n_warps) {
+            unsigned long long best = 0ull;
+            for (int s = lane; s < n_slices; s += 32) {
+                unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x);
+                best = c > best ? c : best;
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+                best = o > best ? o : best;
+            }
+            if (lane == 0) {
+                int32_t tok = (int32_t)best_index(best);
+                toks[x] = tok;
+                a.out_tokens[row0 + x] = tok;
+            }
+        }
+    }
+    sync();
+
+    // empirical distribution: multiplicity of every sampled token within its position
+    for (int x = tid; x < TK; x += nthreads) {
+        const int32_t* row = toks + (x / a.K) * a.K;
+        int32_t y = toks[x];
+        int c = 0;
+        for (int i = 0; i < a.K; ++i) c += (row[i] == y);
+        a.out_counts[row0 + x] = c;
+    }
+
+    if (a.N == 0) {
+        for (int t = tid; t < a.T; t += nthreads) {
+            int hits;
+            bool ok = position_ok(toks + t * a.K, a.K, a.draft[(size_t)b * a.T + t], a.rule, &hits);
+            flag[t] = ok;
+            if (a.out_hits) a.out_hits[(size_t)b * a.T + t] = hits;
+        }
+        sync();
+        if (tid == 0) {
+            int len = 0;
+            while (len < a.T && flag[len]) ++len;   // first rejection ends acceptance
+            a.out_accept_len[b] = len;
+        }
+        sync();   // the scratch may be reused for the next sequence
+        return;
+    }
+
+    // tree: per-node test in parallel, then one serial topological walk
+    const size_t n0 = (size_t)b * a.N;
+    int32_t* depth = flag + a.N;
+    for (int n = tid; n < a.N; n += nthreads) {
+        int h = a.node_hrow[n0 + n];
+        bool ok = false;
+        if (h >= 0 && h < a.T) ok = position_ok(toks + h * a.K, a.K, a.node_token[n0 + n], a.rule, nullptr);
+        flag[n] = ok;
+    }
+    sync();
+    if (tid == 0) {
+        int best_depth = 0, best = -1;
+        for (int n = 0; n < a.N; ++n) {
+            int par = a.node_parent[n0 + n];
+            bool par_ok = par < 0 ? true : (par < n ? flag[par] != 0 : false);
+            int dep = (par < 0 || par >= n) ? 1 : depth[par] + 1;
+            bool ok = par_ok && flag[n];
+            flag[n] = ok;
+            depth[n] = dep;
+            if (ok && dep > best_depth) { best_depth = dep; best = n; }
+        }
+        a.out_accept_len[b] = best_depth;
+        a.out_best_node[b] = best;
+    }
+    sync();
+    if (a.out_node_ok)
+        for (int n = tid; n < a.N; n += nthreads) a.out_node_ok[n0 + n] = flag[n];
+    sync();   // the scratch may be reused for the next sequence
+}
+
+}  // namespace dm

@@ -27,6 +27,7 @@
 // error word, drains and frees TMEM instead of hanging.
 #include <new>
 
+#include "dm_finalize.cuh"
 #include "dm_internal.h"
 #include "dm_ptx.cuh"
 
@@ -69,6 +70,12 @@ struct FusedParams {
     unsigned long long* partials;   // [gridDim.x][rows_total]
     float* dbg_logits;              // [rows_total][V] or null
     uint32_t* err;
+    // When `fold` is set the last CTA to finish also merges the partials and runs the histogram
+    // and the acceptance (a call of one launch): `ticket` counts finished CTAs and is left at 0.
+    int fold;
+    unsigned int* ticket;
+    unsigned long long* best;       // [rows_total], all zero between calls: CTAs reduce into it when folding
+    FinalizeArgs fin;
     // byte offsets into the 1024-aligned dynamic shared memory
     uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar;
 };
@@ -101,6 +108,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int n_bars = 2 * P.nsw + 2 * P.nsb + 2 * P.n_slots;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + n_bars);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+    volatile unsigned int* s_ticket = reinterpret_cast<volatile unsigned int*>(s_tmem + 2);
 
     const int wps = kExpWarps / P.nsb;   // operand-builder warps per ring stage
 
@@ -356,7 +364,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                 unsigned long long c = s_best[w * P.n_pad + n];
                 b = c > b ? c : b;
             }
-            P.partials[(size_t)blockIdx.x * P.rows_total + P.row0 + n] = b;
+            if (P.fold) atomicMax(P.best + P.row0 + n, b);
+            else P.partials[(size_t)blockIdx.x * P.rows_total + P.row0 + n] = b;
         }
         // ------------------------------------------------------------------ teardown
         // Every accumulator has been read, hence every MMA and every TMA load has completed.
@@ -368,6 +377,23 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (warp == kFirstEpiWarp) {
             ptx::tc_fence_after();
             ptx::tmem_dealloc(tmem_base, kTmemCols);
+        }
+        if (P.fold) {
+            // ---------------------------------------------------------------- folded finalize
+            // Whoever draws the last ticket knows that every CTA's partials are in global memory.
+            const int tid_e = threadIdx.x - kFirstEpiWarp * 32;
+            __threadfence();
+            ptx::bar_sync(1, 4 * 32);
+            if (tid_e == 0) *s_ticket = atomicAdd(P.ticket, 1u);
+            ptx::bar_sync(1, 4 * 32);
+            if (*s_ticket == gridDim.x - 1) {
+                __threadfence();
+                int32_t* scratch = reinterpret_cast<int32_t*>(smem + P.off_w);   // the W ring is idle by now
+                for (int b = 0; b < P.fin.B; ++b)
+                    finalize_sequence(P.best, 1, P.rows_total, P.fin, b, scratch, tid_e, 4 * 32, NamedSync{1, 4 * 32});
+                for (int n = tid_e; n < P.rows_total; n += 4 * 32) P.best[n] = 0ull;   // ready for the next call
+                if (tid_e == 0) *P.ticket = 0u;
+            }
         }
     } else {
         if (P.staged) {
@@ -665,7 +691,9 @@ void fused_destroy(FusedState* fs) {
 
 int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hidden*/, int rows,
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
-                 float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out) {
+                 float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
+                 const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out) {
+    if (folded_out) *folded_out = false;
     if (fs == nullptr || !fused_supported(head, rows) || fs->n_ctas > kMaxSlices) return DM_EUNSUPPORTED;
     int launches = 0;
     bool operand_staged = false;
@@ -697,6 +725,12 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.map = map;
         P.key0 = mk.key0; P.key1 = mk.key1; P.thr = mk.thr; P.scale = mk.scale;
         P.partials = partials; P.dbg_logits = dbg_logits; P.err = err;
+        // a call of one launch finishes itself; larger calls leave it to finalize_kernel
+        P.fold = (fin != nullptr && ticket != nullptr && best != nullptr && rows <= kMaxNPad &&
+                  finalize_smem_bytes(fin->T, fin->K, fin->N) <= 32 * 1024) ? 1 : 0;
+        P.ticket = ticket;
+        P.best = best;
+        if (P.fold) { P.fin = *fin; if (folded_out) *folded_out = true; }
         fused_head_kernel<<<fs->n_ctas, kThreads, plan.total, stream>>>(
             fs->tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : fs->tmap_w, P);
         if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;

@@ -61,7 +61,9 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int max_h
 void fused_destroy(FusedState* fs);
 int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidden, int rows,
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
-                 float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out);
+                 float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
+                 const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
+                 unsigned long long* best = nullptr, bool* folded_out = nullptr);
 
 int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo,
                        uint32_t* out_bits, cudaStream_t stream);
