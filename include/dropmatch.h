@@ -101,8 +101,10 @@ int dropmatch_verify_batched(dm_ctx* ctx, const void* H, const int32_t* draft, i
                              int32_t* out_accept_len, void* stream);
 
 /* Same as dropmatch_verify_batched, but H, draft and all outputs are HOST pointers (pinned or
- * pageable).  Copies the inputs to the device, runs the call, copies the outputs back and waits
- * for `stream`.  Needs B*T <= max_hidden_rows of dm_set_head.  out_draft_hits may be NULL. */
+ * pageable).  Gathers the inputs in the context's pinned buffer and sends them with one copy,
+ * runs the call with its outputs going to pinned memory the device can write, waits for
+ * `stream`, and copies the results to the caller's arrays.  Needs B*T <= max_hidden_rows of
+ * dm_set_head.  out_draft_hits may be NULL. */
 int dropmatch_verify_batched_host(dm_ctx* ctx, const void* H_host, const int32_t* draft_host, int B,
                                   int T, int K, float p, uint64_t seed, uint64_t seq_base, int rule,
                                   int32_t* out_tokens_host, int32_t* out_counts_host,

@@ -1,5 +1,6 @@
 // C ABI of libdropmatch: argument checks, workspace, kernel choice.  See include/dropmatch.h.
 #include <math.h>
+#include <string.h>
 #include <new>
 #include <vector>
 
@@ -17,8 +18,13 @@ struct dm_ctx {
     // workspace (device)
     unsigned long long* partials = nullptr;  // [kMaxSlices][max_rows]
     uint32_t* err = nullptr;                 // device error word
-    unsigned char* stage_H = nullptr;        // [max_hidden][d] storage type
-    int32_t* stage_i32 = nullptr;            // draft | tokens | counts | hits | accept_len
+    // staging of the host-buffer entry point: one device buffer and one pinned host buffer with
+    // the same layout, H then the draft tokens; and a pinned, device-mapped buffer that the
+    // kernels write the results into (tokens | counts | hits | accept_len)
+    unsigned char* stage_in = nullptr;       // device
+    unsigned char* pin_in = nullptr;         // pinned host
+    int32_t* pin_out = nullptr;              // pinned host, mapped
+    int32_t* pin_out_dev = nullptr;          // the same memory as the device sees it
     size_t ws_bytes = 0;
     FusedState* fused = nullptr;             // tensor maps etc. of the tcgen05 kernel
     // optional timing of the head kernel alone (dm_profile_head)
@@ -45,8 +51,10 @@ struct DeviceGuard {
 
 void free_workspace(dm_ctx* c) {
     cudaFree(c->partials); c->partials = nullptr;
-    cudaFree(c->stage_H); c->stage_H = nullptr;
-    cudaFree(c->stage_i32); c->stage_i32 = nullptr;
+    cudaFree(c->stage_in); c->stage_in = nullptr;
+    cudaFreeHost(c->pin_in); c->pin_in = nullptr;
+    cudaFreeHost(c->pin_out); c->pin_out = nullptr;
+    c->pin_out_dev = nullptr;
     if (c->fused) { fused_destroy(c->fused); c->fused = nullptr; }
     c->ws_bytes = 0;
 }
@@ -189,17 +197,21 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
     // per-slice partial argmaxes [kMaxSlices][max_rows], then the per-row running best [max_rows]
     // that the fused kernel's CTAs reduce into when one launch covers the call (zero between calls)
     const size_t n_part = ((size_t)kMaxSlices + 1) * max_rows * sizeof(unsigned long long);
-    const size_t n_H = (size_t)max_hidden_rows * d * elem;
-    const size_t n_i32 = ((size_t)3 * max_hidden_rows + 2 * (size_t)max_rows) * sizeof(int32_t);
-    if (cudaMalloc(&c->partials, n_part) != cudaSuccess || cudaMalloc(&c->stage_H, n_H) != cudaSuccess ||
-        cudaMalloc(&c->stage_i32, n_i32) != cudaSuccess ||
+    const size_t n_in = (size_t)max_hidden_rows * d * elem + 16 + (size_t)max_hidden_rows * sizeof(int32_t);
+    const size_t n_out = ((size_t)2 * max_hidden_rows + 2 * (size_t)max_rows) * sizeof(int32_t);
+    void* out_dev = nullptr;
+    if (cudaMalloc(&c->partials, n_part) != cudaSuccess || cudaMalloc(&c->stage_in, n_in) != cudaSuccess ||
+        cudaHostAlloc(reinterpret_cast<void**>(&c->pin_in), n_in, cudaHostAllocDefault) != cudaSuccess ||
+        cudaHostAlloc(reinterpret_cast<void**>(&c->pin_out), n_out, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer(&out_dev, c->pin_out, 0) != cudaSuccess ||
         cudaMemset(c->partials + (size_t)kMaxSlices * max_rows, 0, (size_t)max_rows * sizeof(unsigned long long)) !=
             cudaSuccess) {
         cudaGetLastError();
         free_workspace(c);
         return DM_ECUDA;
     }
-    c->ws_bytes = n_part + n_H + n_i32;
+    c->pin_out_dev = static_cast<int32_t*>(out_dev);
+    c->ws_bytes = n_part + n_in;
     c->head = HeadDesc{W, V, d, dtype};
     c->max_rows = max_rows;
     c->max_hidden = max_hidden_rows;
@@ -262,25 +274,32 @@ int dropmatch_verify_batched_host(dm_ctx* c, const void* H_host, const int32_t* 
     if (!g.ok) return DM_ECUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t elem = c->head.dtype == DM_F32 ? 4 : 2;
-    int32_t* d_draft = c->stage_i32;
-    int32_t* d_hits = d_draft + c->max_hidden;
-    int32_t* d_len = d_hits + c->max_hidden;
-    int32_t* d_tok = d_len + c->max_hidden;
-    int32_t* d_cnt = d_tok + c->max_rows;
-    if (cudaMemcpyAsync(c->stage_H, H_host, (size_t)hidden * c->head.d * elem, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_draft, draft_host, (size_t)hidden * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+    // inputs: gathered in pinned memory, one host-to-device copy
+    const size_t h_bytes = (size_t)hidden * c->head.d * elem;
+    const size_t draft_off = (h_bytes + 15) & ~static_cast<size_t>(15);
+    memcpy(c->pin_in, H_host, h_bytes);
+    memcpy(c->pin_in + draft_off, draft_host, (size_t)hidden * sizeof(int32_t));
+    if (cudaMemcpyAsync(c->stage_in, c->pin_in, draft_off + (size_t)hidden * sizeof(int32_t), cudaMemcpyHostToDevice, s) !=
+        cudaSuccess) {
         cudaGetLastError();
         return DM_ECUDA;
     }
-    st = dropmatch_verify_batched(c, c->stage_H, d_draft, B, T, K, p, seed, seq_base, rule, d_tok, d_cnt,
-                                  d_hits, d_len, stream);
+    // outputs: the kernels write them straight into mapped pinned memory (a few hundred bytes
+    // crossing to the host), so no device-to-host copy has to be queued behind the kernel
+    int32_t* o_tok = c->pin_out;
+    int32_t* o_cnt = o_tok + rows;
+    int32_t* o_hits = o_cnt + rows;
+    int32_t* o_len = o_hits + hidden;
+    int32_t* d_out = c->pin_out_dev;
+    st = dropmatch_verify_batched(c, c->stage_in, reinterpret_cast<const int32_t*>(c->stage_in + draft_off), B, T, K, p,
+                                  seed, seq_base, rule, d_out, d_out + rows, d_out + 2 * rows, d_out + 2 * rows + hidden,
+                                  stream);
     if (st != DM_OK) return st;
-    bool ok = cudaMemcpyAsync(out_tokens_host, d_tok, (size_t)rows * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-              cudaMemcpyAsync(out_counts_host, d_cnt, (size_t)rows * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
-              cudaMemcpyAsync(out_accept_len_host, d_len, (size_t)B * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-    if (ok && out_draft_hits_host)
-        ok = cudaMemcpyAsync(out_draft_hits_host, d_hits, (size_t)hidden * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-    if (!ok || cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    if (cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    memcpy(out_tokens_host, o_tok, (size_t)rows * sizeof(int32_t));
+    memcpy(out_counts_host, o_cnt, (size_t)rows * sizeof(int32_t));
+    memcpy(out_accept_len_host, o_len, (size_t)B * sizeof(int32_t));
+    if (out_draft_hits_host) memcpy(out_draft_hits_host, o_hits, (size_t)hidden * sizeof(int32_t));
     return DM_OK;
 }
 
