@@ -65,21 +65,29 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
             a.out_tokens[row0 + x] = tok;
         }
     } else {
-        for (int x = warp; x < TK; x += n_warps) {
-            unsigned long long best = 0ull;
+        for (int x0 = warp * 4; x0 < TK; x0 += n_warps * 4) {   // four rows at a time: their loads overlap
+            unsigned long long best[4] = {0ull, 0ull, 0ull, 0ull};
             for (int s = lane; s < n_slices; s += 32) {
-                unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x);
-                best = c > best ? c : best;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (x0 + u < TK) {
+                        unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x0 + u);
+                        best[u] = c > best[u] ? c : best[u];
+                    }
+                }
             }
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best, off);
-                best = o > best ? o : best;
-            }
-            if (lane == 0) {
-                int32_t tok = (int32_t)best_index(best);
-                toks[x] = tok;
-                a.out_tokens[row0 + x] = tok;
+            for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+                    unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best[u], off);
+                    best[u] = o > best[u] ? o : best[u];
+                }
+                if (lane == 0 && x0 + u < TK) {
+                    int32_t tok = (int32_t)best_index(best[u]);
+                    toks[x0 + u] = tok;
+                    a.out_tokens[row0 + x0 + u] = tok;
+                }
             }
         }
     }
@@ -119,12 +127,13 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
         bool ok = false;
         if (h >= 0 && h < a.T) ok = position_ok(toks + h * a.K, a.K, a.node_token[n0 + n], a.rule, nullptr);
         flag[n] = ok;
+        depth[n] = a.node_parent[n0 + n];   // staged here so that the serial walk stays in shared memory
     }
     sync();
     if (tid == 0) {
         int best_depth = 0, best = -1;
         for (int n = 0; n < a.N; ++n) {
-            int par = a.node_parent[n0 + n];
+            int par = depth[n];             // still the parent: entries below n already hold depths
             bool par_ok = par < 0 ? true : (par < n ? flag[par] != 0 : false);
             int dep = (par < 0 || par >= n) ? 1 : depth[par] + 1;
             bool ok = par_ok && flag[n];
