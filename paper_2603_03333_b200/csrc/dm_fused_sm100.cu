@@ -10,19 +10,22 @@
 //
 // Loop order.  Tiles are taken in groups of `group_tiles`; inside a group the hidden-size
 // blocks (64 elements = one 128-byte swizzled row) are the outer loop and the tiles the inner
-// one, all accumulators of the group being live at once.  The masked operand of a block is
-// therefore built once per group (once per call when the whole slice fits in TMEM) and reused
-// by every tile of the group, while W still streams through a ring of TMA stages exactly once.
+// one, all accumulators of the group being live at once, while W streams through a ring of
+// TMA stages exactly once.  The masked operand of a block is needed once per group:
+//   - one group (the whole slice fits TMEM): builder warps generate the masks with Philox in
+//     registers and write the masked rows of each block into a shared-memory ring, once per call;
+//   - several groups ("staged"): mask_operand_kernel has written the masked rows to a staging
+//     buffer in global memory once per call, and a second TMA ring streams its blocks in.
 //
 // Warp roles (14 warps):
 //   warp 0      TMA producer: one thread issues cp.async.bulk.tensor loads of W
 //   warp 1      one thread issues tcgen05.mma and the commits
 //   warps 2-5   epilogue: tcgen05.ld the finished accumulators of a group, scale by 1/(1-p),
 //               reduce each column over tiles and lanes to (max, first index), keep the best
-//               per path; warp 2 also allocates and frees TMEM
-//   warps 6-13  operand builders: for every (group, block) write the masked hidden rows into
-//               a swizzled shared-memory ring; mask bytes come from Philox in the first group
-//               and, when they fit, from a shared-memory cache in the later ones
+//               per path; warp 2 also allocates and frees TMEM; the last CTA of a one-launch
+//               call then runs the histogram and the acceptance
+//   warps 6-13  one group: operand builders.  Staged: warps 6-9 are a second set of epilogue
+//               warps, one thread of warp 10 streams the staged operand, the rest retire
 // Rings are guarded by mbarriers; every wait has a time limit after which the CTA sets the
 // error word, drains and frees TMEM instead of hanging.
 #include <new>
@@ -96,7 +99,6 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const uint32_t smem_base = ptx::smem_u32(smem);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* s_bits = smem + P.off_bits;
     RowInfo* s_row = reinterpret_cast<RowInfo*>(smem + P.off_rowinfo);
     unsigned long long* s_best = reinterpret_cast<unsigned long long*>(smem + P.off_best);  // [4][n_pad]
     uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + P.off_bar);
@@ -120,7 +122,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             ptx::mbar_init(b_ready + 8 * s, P.staged ? 1 : wps);
             ptx::mbar_init(b_empty + 8 * s, 1);
         }
-        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, 4); }
+        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, P.staged ? 8 : 4); }
         *s_abort = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
@@ -181,7 +183,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             }
         }
         return;
-    } else if (warp == 1) {
+    }
+    if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane != 0) return;
         const uint32_t idesc = ptx::idesc_bf16_f32(kTileM, P.n_pad);
@@ -237,10 +240,116 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             }
         }
         return;
-    } else if (warp < kFirstExpWarp) {
+    }
+    if (warp >= kFirstExpWarp && P.staged) {
+        if (warp < kFirstExpWarp + 4) {
+            // warps 6-9 have no operand to build: they become a second set of epilogue warps
+        } else {
+            // -------------------------------------------------------------- operand producer
+            // The masked rows were written to the staging buffer by mask_operand_kernel; one
+            // thread streams the [n_pad x 64] block of every (group, block) step through TMA.
+            if (threadIdx.x != (kFirstExpWarp + 4) * 32) return;
+            const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+            uint32_t bar_r = b_ready, bar_e = b_empty, dst = smem_base + P.off_b, parity = 1;
+            int stage = 0;
+            for (int g = 0; g < n_groups; ++g)
+                for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_e, parity, s_abort, kWaitLimitCycles)) {
+                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                        return;
+                    }
+                    ptx::mbar_arrive_expect_tx(bar_r, b_stage_bytes);
+                    ptx::tma_load_2d(dst, &tmap_b, x, P.row0, bar_r);
+                    bar_r += 8; bar_e += 8; dst += b_stage_bytes;
+                    if (++stage == P.nsb) { stage = 0; parity ^= 1; bar_r = b_ready; bar_e = b_empty; dst = smem_base + P.off_b; }
+                }
+            return;
+        }
+    } else if (warp >= kFirstExpWarp) {
+        // ------------------------------------------------------------------ operand builders
+        const int e = warp - kFirstExpWarp;
+        const int grp = e % P.nsb, sub = e / P.nsb;
+        const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+        {   // rows [rows, n_pad) of every stage stay zero for the whole kernel
+            const int tid = threadIdx.x - kFirstExpWarp * 32;
+            uint4* bz = reinterpret_cast<uint4*>(smem + P.off_b);
+            const int n16 = (int)(P.nsb * b_stage_bytes / 16);
+            for (int x = tid; x < n16; x += kExpWarps * 32) bz[x] = make_uint4(0, 0, 0, 0);
+            ptx::fence_proxy_async_smem();
+            ptx::bar_sync(2, kExpWarps * 32);
+        }
+        unsigned char* my_stage = smem + P.off_b + grp * b_stage_bytes;
+        const int n_items = P.rows * 8;            // (row, 16-byte chunk) pairs per block
+        const int stride = wps * 32;               // threads working on this stage
+        const int total_b = n_groups * P.kb_count;
+        for (int m = grp; m < total_b; m += P.nsb) {
+            const int kb = m % P.kb_count;
+            const __nv_bfloat16* h_kb = P.H + kb * kBlockK;
+            // the hidden-state loads do not depend on the stage being free: start them first
+            uint4 hv[4];
+            int it0 = sub * 32 + lane;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int it = it0 + u * stride;
+                if (it < n_items) {
+                    const int q = max(s_row[it >> 3].q, 0);
+                    hv[u] = __ldg(reinterpret_cast<const uint4*>(h_kb + (size_t)q * P.d + (it & 7) * 8));
+                }
+            }
+            if (!ptx::mbar_wait_warp<kPollNs>(b_empty + 8 * grp, ((m / P.nsb) & 1) ^ 1, s_abort,
+                                              kWaitLimitCycles)) {
+                atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                break;
+            }
+            for (; it0 < n_items; it0 += 4 * stride) {
+                // next batch of hidden-state chunks, in flight while this batch is masked
+                uint4 hv_next[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int it = it0 + (4 + u) * stride;
+                    if (it < n_items) {
+                        const int q = max(s_row[it >> 3].q, 0);
+                        hv_next[u] = __ldg(reinterpret_cast<const uint4*>(h_kb + (size_t)q * P.d + (it & 7) * 8));
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int it = it0 + u * stride;
+                    if (it >= n_items) continue;
+                    const int r = it >> 3, c = it & 7;
+                    const RowInfo ri = s_row[r];
+                    RowKey k{0, ri.s, ri.t, ri.i};
+                    const uint32_t quad = (uint32_t)(kb * (kBlockK / 4) + c * 2);
+                    const uint32_t mbits = keep4(quad, k, P.key0, P.key1, P.thr) |
+                                           (keep4(quad + 1, k, P.key0, P.key1, P.thr) << 4);
+                    uint4 o;
+                    o.x = hv[u].x & mask_pair(mbits);
+                    o.y = hv[u].y & mask_pair(mbits >> 2);
+                    o.z = hv[u].z & mask_pair(mbits >> 4);
+                    o.w = hv[u].w & mask_pair(mbits >> 6);
+                    // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
+                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u +
+                                         (uint32_t)((c ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(my_stage + off) = o;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) hv[u] = hv_next[u];
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(b_ready + 8 * grp);
+        }
+        return;
+    }
+
+    {
         // ------------------------------------------------------------------ epilogue
-        const int ew = warp - kFirstEpiWarp;          // row of s_best owned by this warp
-        const int lane_base = (warp & 3) * 32;        // TMEM lanes this warp may read
+        // Warps 2-5, plus warps 6-9 in staged mode, where no operand is built.  Warp w reads TMEM
+        // lanes 32*(w mod 4)..+31; the warps of a lane quarter share the column chunks.
+        const int ew = warp & 3;                      // lane quarter = row of s_best
+        const int set = warp < kFirstExpWarp ? 0 : 1;
+        const int n_sets = P.staged ? 2 : 1;
+        const int lane_base = ew * 32;                // TMEM lanes this warp may read
         // A group's accumulators finish together.  Columns are then taken 16 at a time and, for
         // each, the group's tiles are walked with a per-lane running maximum (a lane always sees
         // increasing vocabulary rows, so a strictly larger value replaces).  Only then are the
@@ -248,7 +357,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // rounds a lane hands half of its packed (key, inverted index) columns to its partner
         // and keeps the maxima of the other half, so that 16 columns cost 16 exchanges, not 80.
         unsigned long long* my_best = s_best + ew * P.n_pad;
-        for (int n = lane; n < P.n_pad; n += 32) my_best[n] = 0ull;
+        for (int n0 = 16 * set; n0 < P.n_pad; n0 += 16 * n_sets)
+            if (lane < 16) my_best[n0 + lane] = 0ull;
         __syncwarp();
         const int m = lane_base + lane;
         const float neg_inf = __uint_as_float(0xFF800000u);
@@ -269,7 +379,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             const int slot0 = t0 % P.n_slots;
             const int v0 = v_cta0 + t0 * P.tile_rows + m;     // this lane's vocabulary row in tile t0
 #pragma unroll 1
-            for (int n0 = 0; n0 < P.n_pad; n0 += 16) {
+            for (int n0 = 16 * set; n0 < P.n_pad; n0 += 16 * n_sets) {
                 float best[16];
                 int bv[16];
 #pragma unroll
@@ -293,17 +403,6 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                                 P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
                                     s_row[n0 + j].q >= 0 ? __uint_as_float(acc[j]) * P.scale
                                                          : __uint_as_float(0x7FC00000u);
-                    }
-                }
-                if (n0 + 16 >= P.n_pad) {   // the group's accumulators are fully read: hand the slots back
-                    ptx::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        int sl = slot0;
-                        for (int tile = t0; tile < t1; ++tile) {
-                            ptx::mbar_arrive(slot_empty + 8 * sl);
-                            if (++sl == P.n_slots) sl = 0;
-                        }
                     }
                 }
                 unsigned long long p16[16];
@@ -354,9 +453,20 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                     if (p1 > my_best[n]) my_best[n] = p1;   // equal keys: the smaller index packs larger
                 }
             }
+            // this warp has read its share of the group's accumulators: hand the slots back
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                int sl = slot0;
+                for (int tile = t0; tile < t1; ++tile) {
+                    ptx::mbar_arrive(slot_empty + 8 * sl);
+                    if (++sl == P.n_slots) sl = 0;
+                }
+            }
         }
-        __syncwarp();
-        ptx::bar_sync(1, 4 * 32);
+        ptx::tc_fence_before();
+        ptx::bar_sync(3, 4 * n_sets * 32);
+        if (warp >= kFirstExpWarp) return;      // the helpers are done; warps 2-5 finish the CTA
         for (int n = threadIdx.x - kFirstEpiWarp * 32; n < P.rows; n += 4 * 32) {
             unsigned long long b = s_best[n];
 #pragma unroll
@@ -394,110 +504,6 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                 for (int n = tid_e; n < P.rows_total; n += 4 * 32) P.best[n] = 0ull;   // ready for the next call
                 if (tid_e == 0) *P.ticket = 0u;
             }
-        }
-    } else {
-        if (P.staged) {
-            // -------------------------------------------------------------- operand producer
-            // The masked rows were written to the staging buffer by mask_operand_kernel; one
-            // thread streams the [n_pad x 64] block of every (group, block) step through TMA.
-            if (threadIdx.x != kFirstExpWarp * 32) return;
-            const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
-            uint32_t bar_r = b_ready, bar_e = b_empty, dst = smem_base + P.off_b, parity = 1;
-            int stage = 0;
-            for (int g = 0; g < n_groups; ++g)
-                for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
-                    if (!ptx::mbar_wait<kPollNs>(bar_e, parity, s_abort, kWaitLimitCycles)) {
-                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
-                        return;
-                    }
-                    ptx::mbar_arrive_expect_tx(bar_r, b_stage_bytes);
-                    ptx::tma_load_2d(dst, &tmap_b, x, P.row0, bar_r);
-                    bar_r += 8; bar_e += 8; dst += b_stage_bytes;
-                    if (++stage == P.nsb) { stage = 0; parity ^= 1; bar_r = b_ready; bar_e = b_empty; dst = smem_base + P.off_b; }
-                }
-            return;
-        }
-        // ------------------------------------------------------------------ operand builders
-        const int e = warp - kFirstExpWarp;
-        const int grp = e % P.nsb, sub = e / P.nsb;
-        const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
-        {   // rows [rows, n_pad) of every stage stay zero for the whole kernel
-            const int tid = threadIdx.x - kFirstExpWarp * 32;
-            uint4* bz = reinterpret_cast<uint4*>(smem + P.off_b);
-            const int n16 = (int)(P.nsb * b_stage_bytes / 16);
-            for (int x = tid; x < n16; x += kExpWarps * 32) bz[x] = make_uint4(0, 0, 0, 0);
-            ptx::fence_proxy_async_smem();
-            ptx::bar_sync(2, kExpWarps * 32);
-        }
-        unsigned char* my_stage = smem + P.off_b + grp * b_stage_bytes;
-        const int n_items = P.rows * 8;            // (row, 16-byte chunk) pairs per block
-        const int bits_pitch = P.d >> 3;           // mask bytes per row
-        const int stride = wps * 32;               // threads working on this stage
-        const int total_b = n_groups * P.kb_count;
-        for (int m = grp; m < total_b; m += P.nsb) {
-            const int g = m / P.kb_count, kb = m - g * P.kb_count;
-            const bool from_cache = P.cache_bits && g > 0;
-            const __nv_bfloat16* h_kb = P.H + kb * kBlockK;
-            // the hidden-state loads do not depend on the stage being free: start them first
-            uint4 hv[4];
-            int it0 = sub * 32 + lane;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int it = it0 + u * stride;
-                if (it < n_items) {
-                    const int q = max(s_row[it >> 3].q, 0);
-                    hv[u] = __ldg(reinterpret_cast<const uint4*>(h_kb + (size_t)q * P.d + (it & 7) * 8));
-                }
-            }
-            if (!ptx::mbar_wait_warp<kPollNs>(b_empty + 8 * grp, ((m / P.nsb) & 1) ^ 1, s_abort,
-                                              kWaitLimitCycles)) {
-                atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
-                break;
-            }
-            for (; it0 < n_items; it0 += 4 * stride) {
-                // next batch of hidden-state chunks, in flight while this batch is masked
-                uint4 hv_next[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int it = it0 + (4 + u) * stride;
-                    if (it < n_items) {
-                        const int q = max(s_row[it >> 3].q, 0);
-                        hv_next[u] = __ldg(reinterpret_cast<const uint4*>(h_kb + (size_t)q * P.d + (it & 7) * 8));
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int it = it0 + u * stride;
-                    if (it >= n_items) continue;
-                    const int r = it >> 3, c = it & 7;
-                    uint32_t mbits;
-                    unsigned char* slot = s_bits + (size_t)r * bits_pitch + kb * 8 + c;
-                    if (from_cache) {
-                        mbits = *slot;
-                    } else {
-                        const RowInfo ri = s_row[r];
-                        RowKey k{0, ri.s, ri.t, ri.i};
-                        const uint32_t quad = (uint32_t)(kb * (kBlockK / 4) + c * 2);
-                        mbits = keep4(quad, k, P.key0, P.key1, P.thr) |
-                                (keep4(quad + 1, k, P.key0, P.key1, P.thr) << 4);
-                        if (P.cache_bits) *slot = (unsigned char)mbits;
-                    }
-                    uint4 o;
-                    o.x = hv[u].x & mask_pair(mbits);
-                    o.y = hv[u].y & mask_pair(mbits >> 2);
-                    o.z = hv[u].z & mask_pair(mbits >> 4);
-                    o.w = hv[u].w & mask_pair(mbits >> 6);
-                    // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
-                    const uint32_t off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u +
-                                         (uint32_t)((c ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4*>(my_stage + off) = o;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) hv[u] = hv_next[u];
-            }
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(b_ready + 8 * grp);
         }
     }
 
