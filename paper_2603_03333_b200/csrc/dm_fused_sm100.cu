@@ -52,6 +52,10 @@ constexpr int kPollNs = 32;                 // pause between polls of a barrier 
 constexpr int kIdlePollNs = 500;            // ... and of one that completes once per tile group
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort flag
+#ifndef DM_PAIR_MIN_NPAD
+#define DM_PAIR_MIN_NPAD 176
+#endif
+constexpr int kPairMinNPad = DM_PAIR_MIN_NPAD;   // staged launches at least this wide run as CTA pairs
 
 struct FusedParams {
     const __nv_bfloat16* H;
@@ -90,6 +94,13 @@ __device__ __forceinline__ uint32_t mask_pair(uint32_t bits2) {
     return ((bits2 & 1u) ? 0x0000FFFFu : 0u) | ((bits2 & 2u) ? 0xFFFF0000u : 0u);
 }
 
+// kPair: the kernel runs as clusters of two CTAs (staged mode only).  Each CTA keeps its own
+// vocabulary slice, W ring, TMEM and epilogue, but loads only half of the operand rows; the
+// leader (cluster rank 0) issues cta_group::2 MMAs that multiply both CTAs' W tiles by the
+// operand rows of both, which halves the operand's shared-memory and L2 traffic per CTA.
+// Barriers that the MMA issuer waits on live in the leader; those that it signals exist in both
+// CTAs and are reached by multicast commits.
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_b,
                   const FusedParams P) {
@@ -107,12 +118,14 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const uint32_t w_full = bar0, w_empty = w_full + 8 * P.nsw;
     const uint32_t b_ready = w_empty + 8 * P.nsw, b_empty = b_ready + 8 * P.nsb;
     const uint32_t slot_full = b_empty + 8 * P.nsb, slot_empty = slot_full + 8 * P.n_slots;
-    const int n_bars = 2 * P.nsw + 2 * P.nsb + 2 * P.n_slots;
+    const int n_bars = 2 * P.nsw + 2 * P.nsb + 2 * P.n_slots + 1;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + n_bars);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
     volatile unsigned int* s_ticket = reinterpret_cast<volatile unsigned int*>(s_tmem + 2);
 
     const int wps = kExpWarps / P.nsb;   // operand-builder warps per ring stage
+    const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;   // 0 = leader of the pair
+    const uint32_t dealloc_bar = slot_empty + 8 * P.n_slots;      // pair only: the other CTA is done with TMEM
 
     if (threadIdx.x == 0) {
         ptx::prefetch_tensormap(&tmap_w);
@@ -122,14 +135,20 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             ptx::mbar_init(b_ready + 8 * s, P.staged ? 1 : wps);
             ptx::mbar_init(b_empty + 8 * s, 1);
         }
-        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, P.staged ? 8 : 4); }
+        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, kPair ? 16 : P.staged ? 8 : 4); }
+        ptx::mbar_init(dealloc_bar, 1);
         *s_abort = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
     }
     if (warp == kFirstEpiWarp) {   // an epilogue warp owns TMEM: it is still whole at the end
-        ptx::tmem_alloc(ptx::smem_u32(s_tmem), kTmemCols);
-        ptx::tmem_relinquish();
+        if (kPair) {
+            ptx::tmem_alloc_pair(ptx::smem_u32(s_tmem), kTmemCols);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(ptx::smem_u32(s_tmem), kTmemCols);
+            ptx::tmem_relinquish();
+        }
     }
     for (int r = threadIdx.x; r < P.rows; r += kThreads) {
         RowKey k;
@@ -139,6 +158,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (kPair) ptx::cluster_sync_all();   // the other CTA's barriers are initialised before anyone signals them
     ptx::tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
 
@@ -148,6 +168,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         my_tiles = (P.V - v_cta0 + P.tile_rows - 1) / P.tile_rows;
         if (my_tiles > P.tiles_per_cta) my_tiles = P.tiles_per_cta;
     }
+    // A pair steps through the same number of tiles: rows past the end of W load as zeros and
+    // are never taken by the epilogue.
+    if (kPair) my_tiles = P.tiles_per_cta;
     const int G = P.group_tiles;
     const int n_groups = (my_tiles + G - 1) / G;
 
@@ -172,8 +195,13 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                         return;
                     }
-                    ptx::mbar_arrive_expect_tx(bar_full, tx_bytes);
-                    ptx::tma_load_2d(dst, &tmap_w, x, v_tile, bar_full);
+                    if (kPair) {   // both tiles of the pair are counted on the leader's barrier
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full, 2 * tx_bytes);
+                        ptx::tma_load_2d_pair(dst, &tmap_w, x, v_tile, ptx::map_to_cta(bar_full, 0));
+                    } else {
+                        ptx::mbar_arrive_expect_tx(bar_full, tx_bytes);
+                        ptx::tma_load_2d(dst, &tmap_w, x, v_tile, bar_full);
+                    }
                     bar_full += 8; bar_empty += 8; dst += kWStageBytes;
                     if (++stage == P.nsw) {
                         stage = 0; empty_parity ^= 1;
@@ -186,9 +214,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     }
     if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane != 0) return;
-        const uint32_t idesc = ptx::idesc_bf16_f32(kTileM, P.n_pad);
-        const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+        if (lane != 0 || rank != 0) return;
+        const uint32_t idesc = ptx::idesc_bf16_f32(kPair ? 2 * kTileM : kTileM, P.n_pad);
+        const uint32_t b_stage_bytes = (uint32_t)(kPair ? P.n_pad / 2 : P.n_pad) * (kBlockK * 2);
         const uint64_t a_desc0 = ptx::smem_desc_sw128(smem_base + P.off_w);
         const uint64_t b_desc0 = ptx::smem_desc_sw128(smem_base + P.off_b);
         // W ring, operand ring and accumulator-slot cursors, all advanced by increments
@@ -222,20 +250,21 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                     ptx::tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
-                        ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-                    ptx::mma_commit(bar_we);
+                        if (kPair) ptx::mma_f16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                        else ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    if (kPair) ptx::mma_commit_pair(bar_we, 3); else ptx::mma_commit(bar_we);
                     bar_wf += 8; bar_we += 8; a_desc += kWStageBytes >> 4;
                     if (++sw == P.nsw) { sw = 0; w_parity ^= 1; bar_wf = w_full; bar_we = w_empty; a_desc = a_desc0; }
                     d_tmem += (uint32_t)P.n_pad;
                     if (++sl == P.n_slots) { sl = 0; d_tmem = tmem_base; }
                 }
-                ptx::mma_commit(bar_be);
+                if (kPair) ptx::mma_commit_pair(bar_be, 3); else ptx::mma_commit(bar_be);
                 bar_br += 8; bar_be += 8; b_desc += b_stage_bytes >> 4;
                 if (++sb == P.nsb) { sb = 0; b_parity ^= 1; bar_br = b_ready; bar_be = b_empty; b_desc = b_desc0; }
             }
             int sl = slot0;
             for (int tile = t0; tile < t1; ++tile) {
-                ptx::mma_commit(slot_full + 8 * sl);
+                if (kPair) ptx::mma_commit_pair(slot_full + 8 * sl, 3); else ptx::mma_commit(slot_full + 8 * sl);
                 if (++sl == P.n_slots) sl = 0;
             }
         }
@@ -249,7 +278,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             // The masked rows were written to the staging buffer by mask_operand_kernel; one
             // thread streams the [n_pad x 64] block of every (group, block) step through TMA.
             if (threadIdx.x != (kFirstExpWarp + 4) * 32) return;
-            const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
+            const int b_rows = kPair ? P.n_pad / 2 : P.n_pad;      // a pair splits the operand rows
+            const int b_row0 = P.row0 + (int)rank * b_rows;
+            const uint32_t b_stage_bytes = (uint32_t)b_rows * (kBlockK * 2);
             uint32_t bar_r = b_ready, bar_e = b_empty, dst = smem_base + P.off_b, parity = 1;
             int stage = 0;
             for (int g = 0; g < n_groups; ++g)
@@ -258,8 +289,13 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                         return;
                     }
-                    ptx::mbar_arrive_expect_tx(bar_r, b_stage_bytes);
-                    ptx::tma_load_2d(dst, &tmap_b, x, P.row0, bar_r);
+                    if (kPair) {
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(bar_r, 2 * b_stage_bytes);
+                        ptx::tma_load_2d_pair(dst, &tmap_b, x, b_row0, ptx::map_to_cta(bar_r, 0));
+                    } else {
+                        ptx::mbar_arrive_expect_tx(bar_r, b_stage_bytes);
+                        ptx::tma_load_2d(dst, &tmap_b, x, b_row0, bar_r);
+                    }
                     bar_r += 8; bar_e += 8; dst += b_stage_bytes;
                     if (++stage == P.nsb) { stage = 0; parity ^= 1; bar_r = b_ready; bar_e = b_empty; dst = smem_base + P.off_b; }
                 }
@@ -458,8 +494,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             __syncwarp();
             if (lane == 0) {
                 int sl = slot0;
-                for (int tile = t0; tile < t1; ++tile) {
-                    ptx::mbar_arrive(slot_empty + 8 * sl);
+                for (int tile = t0; tile < t1; ++tile) {   // the issuer's barrier is the leader's
+                    if (kPair && rank != 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(slot_empty + 8 * sl, 0));
+                    else ptx::mbar_arrive(slot_empty + 8 * sl);
                     if (++sl == P.n_slots) sl = 0;
                 }
             }
@@ -486,7 +523,15 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         ptx::bar_sync(1, 4 * 32);
         if (warp == kFirstEpiWarp) {
             ptx::tc_fence_after();
-            ptx::tmem_dealloc(tmem_base, kTmemCols);
+            if (kPair) {
+                // Neither CTA may free TMEM, or leave, while the other still reads accumulators or
+                // sends signals here: tell the other CTA that this one is done, wait for its word.
+                if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(dealloc_bar, rank ^ 1u));
+                ptx::mbar_wait_warp<kPollNs>(dealloc_bar, 0, s_abort, kWaitLimitCycles);
+                ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+            } else {
+                ptx::tmem_dealloc(tmem_base, kTmemCols);
+            }
         }
         if (P.fold) {
             // ---------------------------------------------------------------- folded finalize
@@ -568,16 +613,23 @@ EncodeTiledFn encode_tiled_fn() {
 
 struct SmemPlan {
     int nsw, nsb, cache_bits, group_tiles, n_slots, staged;
+    int pair;    // run as clusters of two CTAs that split the operand rows
+    int n_pad;   // operand rows after padding: a multiple of 16, of 32 for pairs
     uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar, total;
 };
 
 // Choose the tile grouping, then split the 227 KB of shared memory between the W ring, the
 // operand ring and (only when tiles need more than one group) the mask cache.
-bool plan_smem(int rows, int n_pad, int d, int tiles_per_cta, SmemPlan* out) {
-    (void)rows; (void)d;
+bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     SmemPlan best{};
+    int n_pad = (rows + 15) & ~15;
+    // Staged launches with many operand rows run as CTA pairs: at N >= kPairMinNPad the operand
+    // reads of a lone CTA's MMAs, added to the TMA writes, saturate its shared memory.
+    best.pair = (tiles_per_cta > kTmemCols / n_pad && n_pad >= kPairMinNPad) ? 1 : 0;
+    if (best.pair) n_pad = (rows + 31) & ~31;
+    best.n_pad = n_pad;
     best.n_slots = kTmemCols / n_pad;
-    const uint32_t b_stage = (uint32_t)n_pad * (kBlockK * 2);
+    const uint32_t b_stage = (uint32_t)(best.pair ? n_pad / 2 : n_pad) * (kBlockK * 2);
     const uint32_t fixed = 256u * sizeof(RowInfo) + 4u * n_pad * 8u + kBarBytes;
     const uint32_t avail = kSmemLimit - 1024 - fixed;
     if (tiles_per_cta <= best.n_slots) {
@@ -596,9 +648,13 @@ bool plan_smem(int rows, int n_pad, int d, int tiles_per_cta, SmemPlan* out) {
         const int n_groups = (tiles_per_cta + g - 1) / g;
         best.group_tiles = (tiles_per_cta + n_groups - 1) / n_groups;
         best.staged = 1;
-        // operand ring: up to 96 KB, two to four stages (a stage lasts group_tiles W steps)
+        // operand ring: up to 96 KB in two to eight stages.  Its blocks come from L2 with a
+        // latency of a few microseconds under load and a stage lasts only group_tiles W steps,
+        // so the ring has to be deep, not large.
+        // Pairs (half-height blocks) afford up to eight stages; a lone CTA keeps four at most,
+        // its W ring needs the room more.
         best.nsb = (int)(96u * 1024u / b_stage);
-        if (best.nsb > 4) best.nsb = 4;
+        if (best.nsb > (best.pair ? 8 : 4)) best.nsb = best.pair ? 8 : 4;
         if (best.nsb < 2) best.nsb = 2;
     }
     best.cache_bits = 0;
@@ -657,8 +713,10 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
                         gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { delete fs; return DM_ECUDA; }
-    if (cudaFuncSetAttribute(fused_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
-        cudaSuccess) {
+    if (cudaFuncSetAttribute(fused_head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(fused_head_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
+            cudaSuccess) {
         cudaGetLastError();
         delete fs;
         return DM_ECUDA;
@@ -668,7 +726,7 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
     fs->staging_rows = 0;
     const int widest = max_rows < kMaxNPad ? max_rows : kMaxNPad;
     SmemPlan plan;
-    if (!plan_smem(widest, (widest + 15) & ~15, head.d, fs->tiles_per_cta, &plan)) { delete fs; return DM_EUNSUPPORTED; }
+    if (!plan_smem(widest, fs->tiles_per_cta, &plan)) { delete fs; return DM_EUNSUPPORTED; }
     if (plan.staged) {
         fs->staging_rows = (max_rows + 15) & ~15;
         const size_t n = (size_t)fs->staging_rows * head.d * sizeof(__nv_bfloat16);
@@ -700,7 +758,10 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out) {
     if (folded_out) *folded_out = false;
-    if (fs == nullptr || !fused_supported(head, rows) || fs->n_ctas > kMaxSlices) return DM_EUNSUPPORTED;
+    if (fs == nullptr || !fused_supported(head, rows) || fs->n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
+    // Every launch of a call uses the same even grid (pairs need one); a CTA whose slice lies past
+    // the end of W contributes empty partials.
+    const int grid = (fs->n_ctas + 1) & ~1;
     int launches = 0;
     bool operand_staged = false;
     for (int row0 = 0; row0 < rows; row0 += kMaxNPad) {
@@ -709,11 +770,11 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.d = head.d; P.V = head.V;
         P.rows = rows - row0 < kMaxNPad ? rows - row0 : kMaxNPad;
         P.row0 = row0; P.rows_total = rows;
-        P.n_pad = (P.rows + 15) & ~15;
+        SmemPlan plan;
+        if (!plan_smem(P.rows, fs->tiles_per_cta, &plan)) return DM_EUNSUPPORTED;
+        P.n_pad = plan.n_pad;
         P.kb_count = head.d / kBlockK;
         P.tiles_per_cta = fs->tiles_per_cta; P.tile_rows = fs->tile_rows; P.slice_rows = fs->slice_rows;
-        SmemPlan plan;
-        if (!plan_smem(P.rows, P.n_pad, head.d, fs->tiles_per_cta, &plan)) return DM_EUNSUPPORTED;
         P.group_tiles = plan.group_tiles; P.n_slots = plan.n_slots;
         P.nsw = plan.nsw; P.nsb = plan.nsb; P.cache_bits = plan.cache_bits; P.staged = plan.staged;
         if (plan.staged && !operand_staged) {
@@ -737,12 +798,30 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.ticket = ticket;
         P.best = best;
         if (P.fold) { P.fin = *fin; if (folded_out) *folded_out = true; }
-        fused_head_kernel<<<fs->n_ctas, kThreads, plan.total, stream>>>(
-            fs->tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : fs->tmap_w, P);
+        if (plan.pair) {
+            cudaLaunchConfig_t cfg{};   // clusters of two CTAs
+            cfg.gridDim = dim3((unsigned)grid);
+            cfg.blockDim = dim3(kThreads);
+            cfg.dynamicSmemBytes = plan.total;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr{};
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, fs->tmap_w, fs->tmap_b[P.n_pad / 32 - 1], P) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return DM_ECUDA;
+            }
+        } else {
+            fused_head_kernel<false><<<grid, kThreads, plan.total, stream>>>(
+                fs->tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : fs->tmap_w, P);
+        }
         if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
         ++launches;
     }
-    *n_slices_out = fs->n_ctas;
+    *n_slices_out = grid;
     *launches_out = launches;
     return DM_OK;
 }
