@@ -69,7 +69,6 @@ struct FusedParams {
     int group_tiles;  // tiles whose accumulators are live together
     int n_slots;      // accumulator slots in TMEM (512 / n_pad)
     int nsw, nsb;     // stages of the W ring and of the operand ring
-    int cache_bits;   // keep mask bytes in shared memory after the first group
     int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
     RowMap map;
     uint32_t key0, key1, thr;
@@ -84,7 +83,7 @@ struct FusedParams {
     unsigned long long* best;       // [rows_total], all zero between calls: CTAs reduce into it when folding
     FinalizeArgs fin;
     // byte offsets into the 1024-aligned dynamic shared memory
-    uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar;
+    uint32_t off_w, off_b, off_rowinfo, off_best, off_bar;
 };
 
 struct RowInfo { int q; uint32_t s, t, i; };
@@ -612,14 +611,14 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 struct SmemPlan {
-    int nsw, nsb, cache_bits, group_tiles, n_slots, staged;
+    int nsw, nsb, group_tiles, n_slots, staged;
     int pair;    // run as clusters of two CTAs that split the operand rows
     int n_pad;   // operand rows after padding: a multiple of 16, of 32 for pairs
-    uint32_t off_w, off_b, off_bits, off_rowinfo, off_best, off_bar, total;
+    uint32_t off_w, off_b, off_rowinfo, off_best, off_bar, total;
 };
 
-// Choose the tile grouping, then split the 227 KB of shared memory between the W ring, the
-// operand ring and (only when tiles need more than one group) the mask cache.
+// Choose the operand mode (builders, staged, staged as CTA pairs) and the tile grouping, then
+// split the 227 KB of shared memory between the W ring and the operand ring.
 bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     SmemPlan best{};
     int n_pad = (rows + 15) & ~15;
@@ -657,7 +656,6 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
         if (best.nsb > (best.pair ? 8 : 4)) best.nsb = best.pair ? 8 : 4;
         if (best.nsb < 2) best.nsb = 2;
     }
-    best.cache_bits = 0;
     for (;;) {   // shrink the operand ring until the W ring has six stages (or the ring is at two)
         const uint32_t used = (uint32_t)best.nsb * b_stage;
         if (used + 2u * kWStageBytes <= avail) {
@@ -670,8 +668,7 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     }
     best.off_w = 0;
     best.off_b = (uint32_t)best.nsw * kWStageBytes;
-    best.off_bits = best.off_b + (uint32_t)best.nsb * b_stage;
-    best.off_rowinfo = best.off_bits;
+    best.off_rowinfo = best.off_b + (uint32_t)best.nsb * b_stage;
     best.off_best = best.off_rowinfo + 256u * sizeof(RowInfo);
     best.off_bar = best.off_best + 4u * n_pad * 8u;
     best.total = best.off_bar + kBarBytes + 1024u;
@@ -776,7 +773,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.kb_count = head.d / kBlockK;
         P.tiles_per_cta = fs->tiles_per_cta; P.tile_rows = fs->tile_rows; P.slice_rows = fs->slice_rows;
         P.group_tiles = plan.group_tiles; P.n_slots = plan.n_slots;
-        P.nsw = plan.nsw; P.nsb = plan.nsb; P.cache_bits = plan.cache_bits; P.staged = plan.staged;
+        P.nsw = plan.nsw; P.nsb = plan.nsb; P.staged = plan.staged;
         if (plan.staged && !operand_staged) {
             // one pass over all rows of the call; the launches below read their own rows of it
             if (fs->staging == nullptr || rows > fs->staging_rows) return DM_EWORKSPACE;
@@ -787,7 +784,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
             operand_staged = true;
             ++launches;
         }
-        P.off_w = plan.off_w; P.off_b = plan.off_b; P.off_bits = plan.off_bits;
+        P.off_w = plan.off_w; P.off_b = plan.off_b;
         P.off_rowinfo = plan.off_rowinfo; P.off_best = plan.off_best; P.off_bar = plan.off_bar;
         P.map = map;
         P.key0 = mk.key0; P.key1 = mk.key1; P.thr = mk.thr; P.scale = mk.scale;
