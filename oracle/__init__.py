@@ -75,6 +75,13 @@ def lib() -> ctypes.CDLL:
         L.oracle_verify_tree.argtypes = [vp, ci, ci, ci, vp, i32p, i32p, i32p, ci, ci, ci, ci, cf,
                                          u64, u64, ci, i32p, f64p, i32p, i32p, i32p, i32p]
         L.oracle_verify_tree.restype = None
+        L.oracle_js_divergence.argtypes = [f64p, f64p, ci]
+        L.oracle_js_divergence.restype = ctypes.c_double
+        L.oracle_js_from_logits.argtypes = [f64p, ci, ci, f64p, f64p]
+        L.oracle_js_from_logits.restype = ci
+        L.oracle_verify_js.argtypes = [vp, ci, ci, ci, vp, i32p, ctypes.POINTER(ctypes.c_float), ci, ci, ci, cf,
+                                       u64, u64, i32p, i32p, f64p, i32p, i32p]
+        L.oracle_verify_js.restype = None
         _lib = L
     return _lib
 
@@ -243,3 +250,46 @@ def verify_tree(W, dtype, H, node_token, node_parent, node_hrow, K, p, seed, seq
                              ok.ctypes.data_as(i32p), best.ctypes.data_as(i32p),
                              alen.ctypes.data_as(i32p))
     return dict(tokens=tokens, gap=gap, counts=cnt, node_ok=ok, best_node=best, accept_len=alen)
+
+
+def js_divergence(P, Q) -> float:
+    """Jensen-Shannon divergence (natural logarithm) of two probability vectors."""
+    P = np.ascontiguousarray(P, dtype=np.float64)
+    Q = np.ascontiguousarray(Q, dtype=np.float64)
+    assert P.shape == Q.shape and P.ndim == 1
+    return float(lib().oracle_js_divergence(_f64p(P), _f64p(Q), P.shape[0]))
+
+
+def js_from_logits(logits, draft_prob):
+    """logits[K,V], draft_prob[V] -> (js[K+1], eq5_holds): JS of each head and of the draft to the
+    centroid of Eq. 4."""
+    l = np.ascontiguousarray(logits, dtype=np.float64)
+    dp = np.ascontiguousarray(draft_prob, dtype=np.float64)
+    K, V = l.shape
+    assert dp.shape == (V,)
+    out = np.zeros(K + 1, dtype=np.float64)
+    ok = lib().oracle_js_from_logits(_f64p(l), K, V, _f64p(dp), _f64p(out))
+    return out, bool(ok)
+
+
+def verify_js(W, dtype, H, draft, draft_prob, K, p, seed, seq_base=0):
+    """Algorithm 1 on B chains.  draft_prob[B,T,V] float32.
+    -> dict(tokens[B,T,K], counts, js[B,T,K+1], js_ok[B,T], accept_len[B])."""
+    Ws, Hs = _store(W, dtype), _store(H, dtype)
+    V, d = Ws.shape
+    B, T, d2 = Hs.shape
+    assert d2 == d
+    dr, drp = _i32(draft)
+    dp = np.ascontiguousarray(draft_prob, dtype=np.float32)
+    assert dr.shape == (B, T) and dp.shape == (B, T, V)
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    tokens = np.zeros((B, T, K), dtype=np.int32)
+    cnt = np.zeros((B, T, K), dtype=np.int32)
+    js = np.zeros((B, T, K + 1), dtype=np.float64)
+    js_ok = np.zeros((B, T), dtype=np.int32)
+    alen = np.zeros((B,), dtype=np.int32)
+    lib().oracle_verify_js(Ws.ctypes.data, dtype, V, d, Hs.ctypes.data, drp,
+                           dp.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), B, T, K, float(np.float32(p)), seed,
+                           seq_base, tokens.ctypes.data_as(i32p), cnt.ctypes.data_as(i32p), _f64p(js),
+                           js_ok.ctypes.data_as(i32p), alen.ctypes.data_as(i32p))
+    return dict(tokens=tokens, counts=cnt, js=js, js_ok=js_ok, accept_len=alen)

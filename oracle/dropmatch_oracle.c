@@ -321,3 +321,102 @@ void oracle_verify_tree(const void *W, int dtype, int V, int d, const void *H,
             out_best_node + b);
     }
 }
+
+/* ------------------------------------------------------------------------- */
+/* JS-divergence criterion (Sec. 3.2, Eq. 4, Eq. 5, Algorithm 1)              */
+/* ------------------------------------------------------------------------- */
+
+/* Softmax of V logits, in place into prob[] (max-subtracted, fp64). */
+static void softmax_f64(const double *logits, int V, double *prob)
+{
+    double mx = logits[0];
+    for (int v = 1; v < V; ++v)
+        if (logits[v] > mx) mx = logits[v];
+    double sum = 0.0;
+    for (int v = 0; v < V; ++v) {
+        prob[v] = exp(logits[v] - mx);
+        sum += prob[v];
+    }
+    for (int v = 0; v < V; ++v) prob[v] /= sum;
+}
+
+/* Jensen-Shannon divergence of two distributions over V outcomes, natural
+ * logarithm: JS(P||Q) = KL(P||M)/2 + KL(Q||M)/2 with M = (P+Q)/2; terms with a
+ * zero probability contribute zero. */
+double oracle_js_divergence(const double *P, const double *Q, int V)
+{
+    double acc = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double m = 0.5 * (P[v] + Q[v]);
+        if (P[v] > 0.0) acc += 0.5 * P[v] * log(P[v] / m);
+        if (Q[v] > 0.0) acc += 0.5 * Q[v] * log(Q[v] / m);
+    }
+    return acc;
+}
+
+/* Eq. 4 and both sides of Eq. 5 from explicit logits.  logits[K][V] are the K
+ * head logits of one position, draft_prob[V] the draft model's distribution.
+ * out_js[i] = JS(p^(i) || pbar) for i < K and out_js[K] = JS(phat || pbar),
+ * where pbar = Softmax(mean_i logits[i]) and p^(i) = Softmax(logits[i]).
+ * Returns 1 iff Eq. 5 holds: out_js[K] <= max_i out_js[i]. */
+int oracle_js_from_logits(const double *logits, int K, int V, const double *draft_prob,
+                          double *out_js)
+{
+    double *centroid = (double *)malloc((size_t)V * sizeof(double));
+    double *pbar = (double *)malloc((size_t)V * sizeof(double));
+    double *pi = (double *)malloc((size_t)V * sizeof(double));
+    for (int v = 0; v < V; ++v) {
+        double s = 0.0;
+        for (int i = 0; i < K; ++i) s += logits[(size_t)i * V + v];
+        centroid[v] = s / (double)K;
+    }
+    softmax_f64(centroid, V, pbar);
+    double max_heads = -INFINITY;
+    for (int i = 0; i < K; ++i) {
+        softmax_f64(logits + (size_t)i * V, V, pi);
+        out_js[i] = oracle_js_divergence(pi, pbar, V);
+        if (out_js[i] > max_heads) max_heads = out_js[i];
+    }
+    out_js[K] = oracle_js_divergence(draft_prob, pbar, V);
+    free(centroid);
+    free(pbar);
+    free(pi);
+    return out_js[K] <= max_heads;
+}
+
+/* Algorithm 1 for B chains: per position Eq. 5, else the majority rule of
+ * Eq. 6, else reject; then the left-to-right scan.  draft_prob[B,T,V] is fp32
+ * (the draft model's probabilities), widened exactly.
+ * Outputs: tokens[B,T,K], counts[B,T,K], js[B,T,K+1], js_ok[B,T] (Eq. 5 alone),
+ * accept_len[B]. */
+void oracle_verify_js(const void *W, int dtype, int V, int d, const void *H, const int32_t *draft,
+                      const float *draft_prob, int B, int T, int K, float p, uint64_t seed,
+                      uint64_t seq_base, int32_t *out_tokens, int32_t *out_counts, double *out_js,
+                      int32_t *out_js_ok, int32_t *out_accept_len)
+{
+    const size_t elem = (dtype == ORACLE_F32) ? 4 : 2;
+    double *logits = (double *)malloc((size_t)K * V * sizeof(double));
+    double *dp = (double *)malloc((size_t)V * sizeof(double));
+    for (int b = 0; b < B; ++b) {
+        int len = 0, open = 1;
+        for (int t = 0; t < T; ++t) {
+            const size_t q = (size_t)b * T + t;
+            const void *h_row = (const char *)H + q * d * elem;
+            for (int i = 0; i < K; ++i) {
+                oracle_logits_row(W, dtype, V, d, h_row, p, seed, seq_base + (uint64_t)b, t, i,
+                                  logits + (size_t)i * V);
+                out_tokens[q * K + i] = oracle_argmax(logits + (size_t)i * V, V, NULL);
+            }
+            oracle_counts(out_tokens + q * K, K, draft[q], out_counts + q * K);
+            for (int v = 0; v < V; ++v) dp[v] = (double)draft_prob[q * V + v];
+            int js_ok = oracle_js_from_logits(logits, K, V, dp, out_js + q * (K + 1));
+            out_js_ok[q] = js_ok;
+            int ok = js_ok || oracle_majority_token(out_tokens + q * K, K) == draft[q];
+            if (open && ok) ++len;
+            else open = 0;
+        }
+        out_accept_len[b] = len;
+    }
+    free(logits);
+    free(dp);
+}
