@@ -111,6 +111,28 @@ int dropmatch_verify_batched_host(dm_ctx* ctx, const void* H_host, const int32_t
                                   int32_t* out_draft_hits_host, int32_t* out_accept_len_host,
                                   void* stream);
 
+/* JS-divergence criterion (Sec. 3.2: Eq. 4, Eq. 5, Algorithm 1).  dm_enable_js reserves, after
+ * dm_set_head, the buffers this criterion needs for calls of up to max_rows = B*T*K paths and
+ * max_hidden_rows = B*T positions: fp32 logits of every path (max_rows * V * 4 bytes) and small
+ * partial sums.  Allocates; synchronises the device; a later dm_set_head drops the buffers. */
+int dm_enable_js(dm_ctx* ctx, int max_rows, int max_hidden_rows);
+
+/* Chain verification under Algorithm 1: position t is accepted iff
+ *   JS(phat_t || pbar_t) <= max_i JS(p_t^(i) || pbar_t)                         (Eq. 5), or
+ *   draft[t] is the most frequent of the K path tokens                           (Eq. 6),
+ * where p_t^(i) = Softmax(l_t^(i)), pbar_t = Softmax(mean_i l_t^(i)) (Eq. 4) and phat_t is the
+ * draft model's distribution; then the left-to-right rule.  Natural logarithm; fp32 arithmetic
+ * on fp32 logits.
+ *   draft_prob[B,T,V]   device, fp32 probabilities of the draft model (used as given)
+ *   out_js[B,T,K+1]     device, fp32: JS(p^(i) || pbar) for i < K, then JS(phat || pbar)
+ *   out_js_ok[B,T]      device, 1 iff Eq. 5 holds (may be NULL)
+ *   the rest            as for dropmatch_verify_batched
+ * Needs dm_enable_js with room for the call, else DM_EWORKSPACE.  Only enqueues work. */
+int dropmatch_verify_js(dm_ctx* ctx, const void* H, const int32_t* draft, const float* draft_prob, int B, int T,
+                        int K, float p, uint64_t seed, uint64_t seq_base, int32_t* out_tokens,
+                        int32_t* out_counts, float* out_js, int32_t* out_js_ok, int32_t* out_accept_len,
+                        void* stream);
+
 /* The paper has no counterpart to this entry point; it exists for the way the library gets
  * deployed.  Some hosts of this code cannot ask CUDA for device memory at the time they verify:
  * a serving process that hands all of HBM to its own pool at start-up (a later cudaMalloc fails

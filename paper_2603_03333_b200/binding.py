@@ -33,6 +33,8 @@ SIGNATURES = {
     "dropmatch_verify_batched_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_static": (_ci, [_ci, _vp, _ci, _ci, _ci, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
                                               _vp, _vp, _vp, _vp, _vp]),
+    "dm_enable_js": (_ci, [_vp, _ci, _ci]),
+    "dropmatch_verify_js": (_ci, [_vp, _vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_tree": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
                                     _vp, _vp, _vp, _vp, _vp, _vp]),
     "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
@@ -195,6 +197,25 @@ class Context:
     def alloc_host_outputs(B, T, K, pin=True):
         mk = lambda *s: torch.empty(s, dtype=torch.int32, pin_memory=pin)
         return dict(tokens=mk(B, T, K), counts=mk(B, T, K), hits=mk(B, T), accept_len=mk(B))
+
+    # -- dm_enable_js / dropmatch_verify_js
+    def enable_js(self, max_rows: int, max_hidden_rows: int):
+        _check(lib().dm_enable_js(self._h, max_rows, max_hidden_rows), "dm_enable_js")
+
+    def verify_js(self, H, draft, draft_prob, K, p, seed, seq_base=0):
+        """Algorithm 1 (JS test, else majority).  draft_prob[B,T,V] float32 on the device."""
+        B, T, _ = H.shape
+        _dev(H, self._tdtype(), "H"); _dev(draft, torch.int32, "draft"); _dev(draft_prob, torch.float32, "draft_prob")
+        if tuple(draft_prob.shape) != (B, T, self.V):
+            raise TypeError("draft_prob must have shape [B, T, V]")
+        i32 = dict(dtype=torch.int32, device=self.device)
+        out = dict(tokens=torch.empty((B, T, K), **i32), counts=torch.empty((B, T, K), **i32),
+                   js=torch.empty((B, T, K + 1), dtype=torch.float32, device=self.device),
+                   js_ok=torch.empty((B, T), **i32), accept_len=torch.empty((B,), **i32))
+        _check(lib().dropmatch_verify_js(self._h, _ptr(H), _ptr(draft), _ptr(draft_prob), B, T, K, p, seed, seq_base,
+                                         _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["js"]), _ptr(out["js_ok"]),
+                                         _ptr(out["accept_len"]), _stream(self.device)), "dropmatch_verify_js")
+        return out
 
     # -- dropmatch_verify_tree
     def verify_tree(self, H, node_token, node_parent, node_hrow, K, p, seed, seq_base=0, rule=RULE_NAIVE):

@@ -27,6 +27,10 @@ struct dm_ctx {
     int32_t* pin_out_dev = nullptr;          // the same memory as the device sees it
     size_t ws_bytes = 0;
     FusedState* fused = nullptr;             // tensor maps etc. of the tcgen05 kernel
+    // JS criterion (dm_enable_js): logits of every path of a call, and the kernels' partial sums
+    float* js_logits = nullptr;              // [js_max_rows][V]
+    float* js_ws = nullptr;
+    int js_max_rows = 0, js_max_hidden = 0;
     // optional timing of the head kernel alone (dm_profile_head)
     bool profile = false;
     std::vector<cudaEvent_t> prof_events;    // begin/end pairs, grown on demand
@@ -56,6 +60,9 @@ void free_workspace(dm_ctx* c) {
     cudaFreeHost(c->pin_out); c->pin_out = nullptr;
     c->pin_out_dev = nullptr;
     if (c->fused) { fused_destroy(c->fused); c->fused = nullptr; }
+    cudaFree(c->js_logits); c->js_logits = nullptr;
+    cudaFree(c->js_ws); c->js_ws = nullptr;
+    c->js_max_rows = c->js_max_hidden = 0;
     c->ws_bytes = 0;
 }
 
@@ -86,7 +93,7 @@ int pick_impl(const dm_ctx* c, int rows, int* impl) {
 
 // Masked head + per-slice argmax for `rows` rows, then merge/histogram/acceptance.
 int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const MaskKey& mk,
-               const FinalizeArgs& fa, cudaStream_t stream) {
+               const FinalizeArgs& fa, cudaStream_t stream, float* logits_out = nullptr) {
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
     if (rows > c->max_rows) return DM_EWORKSPACE;
     if (finalize_smem_bytes(fa.T, fa.K, fa.N) > 200 * 1024) return DM_EUNSUPPORTED;
@@ -108,10 +115,10 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
     bool folded = false;
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
-                          nullptr, c->err, stream, &launches, &fa, c->err + 1,
+                          logits_out, c->err, stream, &launches, &fa, c->err + 1,
                           c->partials + (size_t)kMaxSlices * c->max_rows, &folded);
     else {
-        st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, stream);
+        st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, logits_out, c->err, stream);
         launches = 1;
     }
     if (ev_end != nullptr) {
@@ -300,6 +307,63 @@ int dropmatch_verify_batched_host(dm_ctx* c, const void* H_host, const int32_t* 
     memcpy(out_counts_host, o_cnt, (size_t)rows * sizeof(int32_t));
     memcpy(out_accept_len_host, o_len, (size_t)B * sizeof(int32_t));
     if (out_draft_hits_host) memcpy(out_draft_hits_host, o_hits, (size_t)hidden * sizeof(int32_t));
+    return DM_OK;
+}
+
+int dm_enable_js(dm_ctx* c, int max_rows, int max_hidden_rows) {
+    if (c == nullptr) return DM_EINVAL;
+    if (!c->has_head) return DM_ENOHEAD;
+    if (max_rows < 1 || max_hidden_rows < 1 || max_rows > c->max_rows || max_hidden_rows > max_rows) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    cudaFree(c->js_logits); c->js_logits = nullptr;
+    cudaFree(c->js_ws); c->js_ws = nullptr;
+    c->js_max_rows = c->js_max_hidden = 0;
+    const size_t n_logits = (size_t)max_rows * c->head.V * sizeof(float);
+    const size_t n_ws = js_workspace_floats(c->head.V, max_rows, max_hidden_rows) * sizeof(float);
+    if (cudaMalloc(&c->js_logits, n_logits) != cudaSuccess || cudaMalloc(&c->js_ws, n_ws) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(c->js_logits); c->js_logits = nullptr;
+        cudaFree(c->js_ws); c->js_ws = nullptr;
+        return DM_ECUDA;
+    }
+    c->js_max_rows = max_rows;
+    c->js_max_hidden = max_hidden_rows;
+    c->ws_bytes += n_logits + n_ws;
+    return DM_OK;
+}
+
+int dropmatch_verify_js(dm_ctx* c, const void* H, const int32_t* draft, const float* draft_prob, int B, int T,
+                        int K, float p, uint64_t seed, uint64_t seq_base, int32_t* out_tokens,
+                        int32_t* out_counts, float* out_js, int32_t* out_js_ok, int32_t* out_accept_len,
+                        void* stream) {
+    int st = check_common(c, H, B, T, K);
+    if (st != DM_OK) return st;
+    if (draft == nullptr || draft_prob == nullptr || out_tokens == nullptr || out_counts == nullptr ||
+        out_js == nullptr || out_accept_len == nullptr)
+        return DM_EINVAL;
+    const long long hidden = (long long)B * T, rows = hidden * K;
+    if (c->js_logits == nullptr || rows > c->js_max_rows || hidden > c->js_max_hidden) return DM_EWORKSPACE;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the ordinary call (tokens, counts; its own accepted length is the majority rule's and is
+    // overwritten below) with every logit of every path kept in the context's buffer
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base};
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = T; fa.K = K; fa.rule = DM_RULE_MAJORITY;
+    fa.draft = draft; fa.out_hits = nullptr;
+    fa.N = 0;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    st = run_verify(c, H, (int)rows, map, mk, fa, s, c->js_logits);
+    if (st != DM_OK) return st;
+    st = launch_js(c->js_logits, draft_prob, c->js_ws, c->head.V, B, T, K, out_tokens, draft, out_js, out_js_ok,
+                   out_accept_len, s);
+    if (st != DM_OK) return st;
+    c->last_launches += 3;
     return DM_OK;
 }
 

@@ -65,6 +65,13 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidd
                  const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
                  unsigned long long* best = nullptr, bool* folded_out = nullptr);
 
+// JS-divergence acceptance (Eq. 4, Eq. 5, Algorithm 1) on logits [B*T*K][V] written by a head kernel.
+int js_chunks(int V);
+size_t js_workspace_floats(int V, int max_rows, int max_hidden);
+int launch_js(const float* logits, const float* draft_prob, float* workspace, int V, int B, int T, int K,
+              const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
+              int32_t* out_accept_len, cudaStream_t stream);
+
 int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo,
                        uint32_t* out_bits, cudaStream_t stream);
 

@@ -1,0 +1,186 @@
+// JS-divergence acceptance (Sec. 3.2: Eq. 4 centroid, Eq. 5 test, Algorithm 1) on the logits that
+// a head kernel has written to global memory.  Three small kernels over [n_pos][K][V] fp32
+// logits (20 MB for the Llama-3-8B head at 40 paths, L2-resident right after the head kernel):
+//   js_lse_kernel      per (position, vocabulary chunk): partial log-sum-exp of each of the K
+//                      paths and of the centroid logits (their mean over the paths)
+//   js_sum_kernel      per (position, chunk): merges the partial log-sum-exps, then the chunk's
+//                      share of JS(p_i || pbar) for every path and of JS(phat || pbar)
+//   js_accept_kernel   per sequence: sums the shares, Eq. 5, else Eq. 6, left-to-right scan
+// Probabilities are never stored: p = exp(l - lse) is recomputed where it is needed.
+#include "dm_finalize.cuh"
+#include "dm_internal.h"
+
+namespace dm {
+
+namespace {
+
+constexpr int kJsThreads = 256;
+
+__device__ __forceinline__ float block_reduce_sum(float x, float* red) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, off);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    float t = 0.0f;
+    for (int w = 0; w < kJsThreads / 32; ++w) t += red[w];
+    return t;
+}
+__device__ __forceinline__ float block_reduce_max(float x, float* red) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x = fmaxf(x, __shfl_xor_sync(0xFFFFFFFFu, x, off));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    float t = red[0];
+    for (int w = 1; w < kJsThreads / 32; ++w) t = fmaxf(t, red[w]);
+    return t;
+}
+
+// Logit of series s at vocabulary entry v of one position: path s for s < K, else the centroid.
+__device__ __forceinline__ float series_logit(const float* __restrict__ pos_logits, int V, int K, int s, int v) {
+    if (s < K) return pos_logits[(size_t)s * V + v];
+    float acc = 0.0f;
+    for (int i = 0; i < K; ++i) acc += pos_logits[(size_t)i * V + v];
+    return acc / (float)K;
+}
+
+// part[(pos*(K+1) + s)*n_chunks + chunk] = (max, sum of exp(l - max)) over the chunk
+__global__ void __launch_bounds__(kJsThreads)
+js_lse_kernel(const float* __restrict__ logits, int V, int K, int chunk_len, int n_chunks,
+              float2* __restrict__ part) {
+    extern __shared__ float cen[];   // [chunk_len] centroid logits of the chunk (Eq. 4 before the softmax)
+    __shared__ float red[kJsThreads / 32];
+    const int pos = blockIdx.y, chunk = blockIdx.x;
+    const int v0 = chunk * chunk_len, v1 = min(V, v0 + chunk_len);
+    const float* pl = logits + (size_t)pos * K * V;
+    for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) cen[v - v0] = series_logit(pl, V, K, K, v);
+    __syncthreads();
+    for (int s = 0; s <= K; ++s) {
+        float mx = -INFINITY;
+        for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads)
+            mx = fmaxf(mx, s < K ? pl[(size_t)s * V + v] : cen[v - v0]);
+        mx = block_reduce_max(mx, red);
+        float sum = 0.0f;
+        for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads)
+            sum += expf((s < K ? pl[(size_t)s * V + v] : cen[v - v0]) - mx);
+        sum = block_reduce_sum(sum, red);
+        if (threadIdx.x == 0) part[((size_t)pos * (K + 1) + s) * n_chunks + chunk] = make_float2(mx, sum);
+    }
+}
+
+// One term of 2*JS(P||Q) at an outcome with log-probabilities lp, lq (natural logarithm):
+// P log(P/M) + Q log(Q/M), M = (P+Q)/2.  A vanishing probability contributes nothing.
+// Written around the log-ratio a = lo - hi <= 0 of the smaller to the larger probability, so that
+// nothing is lost to cancellation between large log-probabilities: log(hi/M) = -log((1+e^a)/2).
+__device__ __forceinline__ float js_term(float lp, float lq) {
+    const float hi = fmaxf(lp, lq), lo = fminf(lp, lq);
+    if (hi == -INFINITY) return 0.0f;
+    const float a = lo - hi;                                  // may be -inf
+    const float r = -logf(0.5f + 0.5f * expf(a));             // log(P_hi / M), in [0, log 2]
+    float t = expf(hi) * r;
+    if (a > -INFINITY) t += expf(lo) * (a + r);               // log(P_lo / M) = a + r
+    return t;
+}
+
+// share[(pos*(K+1) + s)*n_chunks + chunk] = this chunk's part of JS(series s || centroid) for
+// s < K, and of JS(draft || centroid) for s = K.
+__global__ void __launch_bounds__(kJsThreads)
+js_sum_kernel(const float* __restrict__ logits, const float* __restrict__ draft_prob, int V, int K, int chunk_len,
+              int n_chunks, const float2* __restrict__ part, float* __restrict__ share) {
+    extern __shared__ float js_smem[];
+    float* lse = js_smem;            // [K+1]
+    float* lqs = js_smem + K + 1;    // [chunk_len] log pbar of the chunk
+    __shared__ float red[kJsThreads / 32];
+    const int pos = blockIdx.y, chunk = blockIdx.x;
+    for (int s = threadIdx.x; s <= K; s += kJsThreads) {
+        const float2* ps = part + ((size_t)pos * (K + 1) + s) * n_chunks;
+        float mx = -INFINITY;
+        for (int c = 0; c < n_chunks; ++c) mx = fmaxf(mx, ps[c].x);
+        float sum = 0.0f;
+        for (int c = 0; c < n_chunks; ++c) sum += ps[c].y * expf(ps[c].x - mx);
+        lse[s] = mx + logf(sum);
+    }
+    __syncthreads();
+    const int v0 = chunk * chunk_len, v1 = min(V, v0 + chunk_len);
+    const float* pl = logits + (size_t)pos * K * V;
+    const float* dp = draft_prob + (size_t)pos * V;
+    const float lse_c = lse[K];
+    for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) lqs[v - v0] = series_logit(pl, V, K, K, v) - lse_c;
+    __syncthreads();
+    for (int s = 0; s <= K; ++s) {
+        float acc = 0.0f;
+        for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) {
+            float lp;
+            if (s < K) lp = pl[(size_t)s * V + v] - lse[s];                   // log p_s[v]
+            else { const float P = dp[v]; lp = P > 0.0f ? logf(P) : -INFINITY; }
+            acc += js_term(lp, lqs[v - v0]);
+        }
+        acc = block_reduce_sum(acc, red);
+        if (threadIdx.x == 0) share[((size_t)pos * (K + 1) + s) * n_chunks + chunk] = 0.5f * acc;
+    }
+}
+
+// Algorithm 1 and the left-to-right scan for one sequence; also exports the divergences.
+__global__ void __launch_bounds__(kJsThreads)
+js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, const int32_t* __restrict__ tokens,
+                 const int32_t* __restrict__ draft, float* __restrict__ out_js, int32_t* __restrict__ out_js_ok,
+                 int32_t* __restrict__ out_accept_len) {
+    extern __shared__ int32_t ok[];   // [T]
+    const int b = blockIdx.x;
+    // divergences: one thread per (position, series), chunks summed in double
+    for (int x = threadIdx.x; x < T * (K + 1); x += kJsThreads) {
+        const size_t idx = (size_t)b * T * (K + 1) + x;
+        double acc = 0.0;
+        for (int c = 0; c < n_chunks; ++c) acc += (double)share[idx * n_chunks + c];
+        out_js[idx] = (float)acc;
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < T; t += kJsThreads) {
+        const size_t q = (size_t)b * T + t;
+        const float* js = out_js + q * (K + 1);
+        float max_heads = js[0];
+        for (int i = 1; i < K; ++i) max_heads = fmaxf(max_heads, js[i]);
+        const bool eq5 = js[K] <= max_heads;                                   // Eq. 5
+        const bool eq6 = position_ok(tokens + q * K, K, draft[q], DM_RULE_MAJORITY, nullptr);   // Eq. 6
+        if (out_js_ok) out_js_ok[q] = eq5;
+        ok[t] = eq5 || eq6;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int len = 0;
+        while (len < T && ok[len]) ++len;
+        out_accept_len[b] = len;
+    }
+}
+
+}  // namespace
+
+int js_chunks(int V) {
+    const int n = (V + 4095) / 4096;
+    return n < 1 ? 1 : n;
+}
+
+size_t js_workspace_floats(int V, int max_rows, int max_hidden) {
+    // partial (max, sum) pairs and JS shares for every (position, series, chunk)
+    return (size_t)(max_rows + max_hidden) * js_chunks(V) * 3;
+}
+
+int launch_js(const float* logits, const float* draft_prob, float* workspace, int V, int B, int T, int K,
+              const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
+              int32_t* out_accept_len, cudaStream_t stream) {
+    const int n_pos = B * T, n_chunks = js_chunks(V);
+    const int chunk_len = (V + n_chunks - 1) / n_chunks;
+    float2* part = reinterpret_cast<float2*>(workspace);
+    float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
+    if ((size_t)(K + 1 + chunk_len) * sizeof(float) > 40 * 1024 || (size_t)T * sizeof(int32_t) > 40 * 1024) return DM_EUNSUPPORTED;
+    dim3 grid((unsigned)n_chunks, (unsigned)n_pos);
+    js_lse_kernel<<<grid, kJsThreads, chunk_len * sizeof(float), stream>>>(logits, V, K, chunk_len, n_chunks, part);
+    js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K, chunk_len,
+                                                                      n_chunks, part, share);
+    js_accept_kernel<<<B, kJsThreads, T * sizeof(int32_t), stream>>>(share, n_chunks, T, K, tokens, draft, out_js,
+                                                                  out_js_ok, out_accept_len);
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+}
+
+}  // namespace dm

@@ -119,6 +119,21 @@ def make_chain_draft(topk: torch.Tensor, B: int, T: int, V: int, mode: str, seed
     return torch.from_numpy(draft)
 
 
+def make_draft_probs(W: torch.Tensor, H: torch.Tensor, noise, seed: int = 6) -> torch.Tensor:
+    """draft_prob[n_rows,V] float32: a stand-in for the draft model's distribution, the softmax of
+    the plain (undropped) head applied to H + noise * N(0,1); ``noise`` is a float or one value per
+    row (small: the draft agrees with the target; large: it does not).  Library matmul/softmax."""
+    g = _gen(seed, H.device)
+    Hf = H.to(torch.float32)
+    n = torch.as_tensor(noise, dtype=torch.float32, device=H.device).reshape(-1, 1)
+    Hn = Hf + n * torch.randn(Hf.shape, generator=g, device=H.device, dtype=torch.float32)
+    out = torch.empty((H.shape[0], W.shape[0]), dtype=torch.float32, device=H.device)
+    step = 32
+    for r0 in range(0, H.shape[0], step):
+        out[r0:r0 + step] = torch.softmax(Hn[r0:r0 + step] @ W.to(torch.float32).T, dim=1)
+    return out
+
+
 def make_tree_shape(B: int, N: int, max_depth: int = 7, max_branch: int = 4, seed: int = 4):
     """Random draft trees in topological order.
 
