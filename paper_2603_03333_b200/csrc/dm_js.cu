@@ -157,7 +157,7 @@ js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, co
 }  // namespace
 
 int js_chunks(int V) {
-    const int n = (V + 4095) / 4096;
+    const int n = (V + 1023) / 1024;   // short chunks: several hundred blocks even for a handful of positions
     return n < 1 ? 1 : n;
 }
 
