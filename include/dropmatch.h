@@ -59,6 +59,7 @@ enum {
 enum { DM_F32 = 0, DM_BF16 = 1 };             /* storage type of W and H (accumulation is fp32) */
 enum { DM_RULE_NAIVE = 0, DM_RULE_MAJORITY = 1 };
 enum { DM_IMPL_AUTO = 0, DM_IMPL_SIMT = 1, DM_IMPL_TCGEN05 = 2 };
+enum { DM_MASK_PER_POSITION = 0, DM_MASK_PER_PATH = 1 };
 
 /* Create a context on CUDA device `device` (must be sm_100).  *out is set on success. */
 int dm_create(dm_ctx** out, int device);
@@ -77,6 +78,13 @@ int dm_set_head(dm_ctx* ctx, const void* W, int V, int d, int dtype, int max_row
 /* Force a kernel family (DM_IMPL_*) for later calls; DM_IMPL_AUTO restores the default choice.
  * DM_IMPL_TCGEN05 on a head it cannot handle makes verify calls return DM_EUNSUPPORTED. */
 int dm_set_impl(dm_ctx* ctx, int impl);
+
+/* How Eq. 1's masks are keyed for later calls.  DM_MASK_PER_POSITION (default): an independent
+ * mask per (sequence, position, path).  DM_MASK_PER_PATH: the position is left out of the key, so
+ * path i of a sequence applies one and the same mask m^(i) at every position (for trees: at every
+ * hidden row) -- the K paths then behave as K persistent heads, which is how Eq. 1 and the
+ * per-head table of Sec. 3.1 can also be read.  Everything else is unchanged. */
+int dm_set_mask_mode(dm_ctx* ctx, int mode);
 
 /* Verify one chain of T draft tokens (sequence id 0): Eq. 1-3, per-path argmax, token counts,
  * acceptance scan.

@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_verify_batched.argtypes = [vp, ci, ci, ci, vp, i32p, ci, ci, ci, cf, u64, u64, ci,
                                             i32p, f64p, i32p, i32p, i32p]
         L.oracle_verify_batched.restype = None
+        L.oracle_verify_batched_ex.argtypes = [vp, ci, ci, ci, vp, i32p, ci, ci, ci, cf, u64, u64, ci, ci,
+                                               i32p, f64p, i32p, i32p, i32p]
+        L.oracle_verify_batched_ex.restype = None
         L.oracle_verify_tree.argtypes = [vp, ci, ci, ci, vp, i32p, i32p, i32p, ci, ci, ci, ci, cf,
                                          u64, u64, ci, i32p, f64p, i32p, i32p, i32p, i32p]
         L.oracle_verify_tree.restype = None
@@ -204,8 +207,9 @@ def accept_tree(tokens, node_token, node_parent, node_hrow, rule=RULE_NAIVE):
     return int(L), int(best.value), ok[:N]
 
 
-def verify_batched(W, dtype, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE):
-    """H[B,T,d], draft[B,T] -> dict(tokens[B,T,K], gap, counts, hits[B,T], accept_len[B])."""
+def verify_batched(W, dtype, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE, shared_masks=False):
+    """H[B,T,d], draft[B,T] -> dict(tokens[B,T,K], gap, counts, hits[B,T], accept_len[B]).
+    shared_masks: one mask per (sequence, path) for all positions instead of one per position."""
     Ws, Hs = _store(W, dtype), _store(H, dtype)
     V, d = Ws.shape
     B, T, d2 = Hs.shape
@@ -218,9 +222,9 @@ def verify_batched(W, dtype, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE):
     cnt = np.zeros((B, T, K), dtype=np.int32)
     hits = np.zeros((B, T), dtype=np.int32)
     alen = np.zeros((B,), dtype=np.int32)
-    lib().oracle_verify_batched(Ws.ctypes.data, dtype, V, d, Hs.ctypes.data, drp, B, T, K,
-                                float(np.float32(p)), seed, seq_base, rule,
-                                tokens.ctypes.data_as(i32p), _f64p(gap), cnt.ctypes.data_as(i32p),
+    lib().oracle_verify_batched_ex(Ws.ctypes.data, dtype, V, d, Hs.ctypes.data, drp, B, T, K,
+                                   float(np.float32(p)), seed, seq_base, rule, int(bool(shared_masks)),
+                                   tokens.ctypes.data_as(i32p), _f64p(gap), cnt.ctypes.data_as(i32p),
                                 hits.ctypes.data_as(i32p), alen.ctypes.data_as(i32p))
     return dict(tokens=tokens, gap=gap, counts=cnt, hits=hits, accept_len=alen)
 

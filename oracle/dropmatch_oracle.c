@@ -262,13 +262,14 @@ int oracle_accept_tree(const int32_t *tokens /*[N_h,K]*/, const int32_t *node_to
  * path (q, i) is written at out_tokens[q*K + i]. */
 static void sample_tokens(const void *W, int dtype, int V, int d, const void *H, int n_bt,
                           int rows_per_seq, int K, float p, uint64_t seed, uint64_t seq_base,
-                          int32_t *out_tokens, double *out_gap)
+                          int shared_masks, int32_t *out_tokens, double *out_gap)
 {
     const size_t elem = (dtype == ORACLE_F32) ? 4 : 2;
     double *logits = (double *)malloc((size_t)V * sizeof(double));
     for (int q = 0; q < n_bt; ++q) {
         const uint64_t s = seq_base + (uint64_t)(q / rows_per_seq);
-        const int t = q % rows_per_seq;
+        /* shared masks: path i uses one mask m^(i) at every position, i.e. position 0's key */
+        const int t = shared_masks ? 0 : q % rows_per_seq;
         const void *h_row = (const char *)H + (size_t)q * d * elem;
         for (int i = 0; i < K; ++i) {
             double gap;
@@ -280,15 +281,18 @@ static void sample_tokens(const void *W, int dtype, int V, int d, const void *H,
     free(logits);
 }
 
-/* Chain verification of B independent sequences (sequence b has id seq_base+b).
+/* shared_masks = 1 is the other reading of Eq. 1 (m^(i) carries no position index): the K paths
+ * are K persistent heads, each with one mask for all positions of a sequence.
+ * Chain verification of B independent sequences (sequence b has id seq_base+b).
  * H[B,T,d], draft[B,T] -> tokens[B,T,K], gap[B,T,K] (may be NULL),
  * counts[B,T,K], hits[B,T], accept_len[B]. */
-void oracle_verify_batched(const void *W, int dtype, int V, int d, const void *H,
-                           const int32_t *draft, int B, int T, int K, float p, uint64_t seed,
-                           uint64_t seq_base, int rule, int32_t *out_tokens, double *out_gap,
-                           int32_t *out_counts, int32_t *out_hits, int32_t *out_accept_len)
+void oracle_verify_batched_ex(const void *W, int dtype, int V, int d, const void *H,
+                              const int32_t *draft, int B, int T, int K, float p, uint64_t seed,
+                              uint64_t seq_base, int rule, int shared_masks, int32_t *out_tokens,
+                              double *out_gap, int32_t *out_counts, int32_t *out_hits,
+                              int32_t *out_accept_len)
 {
-    sample_tokens(W, dtype, V, d, H, B * T, T, K, p, seed, seq_base, out_tokens, out_gap);
+    sample_tokens(W, dtype, V, d, H, B * T, T, K, p, seed, seq_base, shared_masks, out_tokens, out_gap);
     for (int b = 0; b < B; ++b) {
         for (int t = 0; t < T; ++t) {
             size_t q = (size_t)b * T + t;
@@ -300,6 +304,16 @@ void oracle_verify_batched(const void *W, int dtype, int V, int d, const void *H
     }
 }
 
+/* The default reading (R1): an independent mask per (sequence, position, path). */
+void oracle_verify_batched(const void *W, int dtype, int V, int d, const void *H,
+                           const int32_t *draft, int B, int T, int K, float p, uint64_t seed,
+                           uint64_t seq_base, int rule, int32_t *out_tokens, double *out_gap,
+                           int32_t *out_counts, int32_t *out_hits, int32_t *out_accept_len)
+{
+    oracle_verify_batched_ex(W, dtype, V, d, H, draft, B, T, K, p, seed, seq_base, rule, 0, out_tokens,
+                             out_gap, out_counts, out_hits, out_accept_len);
+}
+
 /* Tree verification of B sequences: H[B,N_h,d]; per sequence N nodes
  * (token, parent, hrow).  counts are multiplicities per hidden row. */
 void oracle_verify_tree(const void *W, int dtype, int V, int d, const void *H,
@@ -309,7 +323,7 @@ void oracle_verify_tree(const void *W, int dtype, int V, int d, const void *H,
                         double *out_gap, int32_t *out_counts, int32_t *out_node_ok,
                         int32_t *out_best_node, int32_t *out_accept_len)
 {
-    sample_tokens(W, dtype, V, d, H, B * N_h, N_h, K, p, seed, seq_base, out_tokens, out_gap);
+    sample_tokens(W, dtype, V, d, H, B * N_h, N_h, K, p, seed, seq_base, 0, out_tokens, out_gap);
     for (int b = 0; b < B; ++b) {
         for (int q = 0; q < N_h; ++q) {
             size_t row = (size_t)b * N_h + q;

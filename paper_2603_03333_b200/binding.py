@@ -16,6 +16,7 @@ STATIC_MAX_ROWS = 256
 F32, BF16 = 0, 1
 RULE_NAIVE, RULE_MAJORITY = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+MASK_PER_POSITION, MASK_PER_PATH = 0, 1
 
 _LIB_PATH = Path(__file__).resolve().parent / "libdropmatch.so"
 _lib = None
@@ -28,6 +29,7 @@ SIGNATURES = {
     "dm_destroy": (_ci, [_vp]),
     "dm_set_head": (_ci, [_vp, _vp, _ci, _ci, _ci, _ci, _ci]),
     "dm_set_impl": (_ci, [_vp, _ci]),
+    "dm_set_mask_mode": (_ci, [_vp, _ci]),
     "dropmatch_verify": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _u64, _ci, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
@@ -148,6 +150,9 @@ class Context:
 
     def set_impl(self, impl: int):
         _check(lib().dm_set_impl(self._h, impl), "dm_set_impl")
+
+    def set_mask_mode(self, mode: int):
+        _check(lib().dm_set_mask_mode(self._h, mode), "dm_set_mask_mode")
 
     # -- dropmatch_verify
     def verify(self, H, draft, K, p, seed, rule=RULE_NAIVE):

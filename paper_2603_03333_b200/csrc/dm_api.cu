@@ -14,6 +14,7 @@ struct dm_ctx {
     bool has_head = false;
     int max_rows = 0, max_hidden = 0;
     int impl = DM_IMPL_AUTO;
+    int mask_mode = DM_MASK_PER_POSITION;
     int last_impl = 0, last_launches = 0;
     // workspace (device)
     unsigned long long* partials = nullptr;  // [kMaxSlices][max_rows]
@@ -236,6 +237,12 @@ int dm_set_impl(dm_ctx* c, int impl) {
     return DM_OK;
 }
 
+int dm_set_mask_mode(dm_ctx* c, int mode) {
+    if (c == nullptr || (mode != DM_MASK_PER_POSITION && mode != DM_MASK_PER_PATH)) return DM_EINVAL;
+    c->mask_mode = mode;
+    return DM_OK;
+}
+
 int dropmatch_verify_batched(dm_ctx* c, const void* H, const int32_t* draft, int B, int T, int K,
                              float p, uint64_t seed, uint64_t seq_base, int rule, int32_t* out_tokens,
                              int32_t* out_counts, int32_t* out_draft_hits, int32_t* out_accept_len,
@@ -249,7 +256,7 @@ int dropmatch_verify_batched(dm_ctx* c, const void* H, const int32_t* draft, int
     if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
-    RowMap map{nullptr, K, T, B, (uint32_t)seq_base};
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};
     FinalizeArgs fa{};
     fa.B = B; fa.T = T; fa.K = K; fa.rule = rule;
     fa.draft = draft; fa.out_hits = out_draft_hits;
@@ -352,7 +359,7 @@ int dropmatch_verify_js(dm_ctx* c, const void* H, const int32_t* draft, const fl
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the ordinary call (tokens, counts; its own accepted length is the majority rule's and is
     // overwritten below) with every logit of every path kept in the context's buffer
-    RowMap map{nullptr, K, T, B, (uint32_t)seq_base};
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};
     FinalizeArgs fa{};
     fa.B = B; fa.T = T; fa.K = K; fa.rule = DM_RULE_MAJORITY;
     fa.draft = draft; fa.out_hits = nullptr;
@@ -383,7 +390,7 @@ int dropmatch_verify_tree(dm_ctx* c, const void* H, const int32_t* node_token, c
     if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
-    RowMap map{nullptr, K, N_h, B, (uint32_t)seq_base};
+    RowMap map{nullptr, K, N_h, B, (uint32_t)seq_base, c->mask_mode};
     FinalizeArgs fa{};
     fa.B = B; fa.T = N_h; fa.K = K; fa.rule = rule;
     fa.N = N; fa.node_token = node_token; fa.node_parent = node_parent; fa.node_hrow = node_hrow;
@@ -404,7 +411,7 @@ int dm_debug_logits(dm_ctx* c, const void* H, int B, int T, const int32_t* row_s
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
-    RowMap map{row_sel, 1, T, B, (uint32_t)seq_base};
+    RowMap map{row_sel, 1, T, B, (uint32_t)seq_base, c->mask_mode};
     int impl;
     int st = pick_impl(c, n_sel, &impl);
     if (st != DM_OK) return st;
@@ -430,7 +437,7 @@ int dm_debug_masks(dm_ctx* c, int B, int T, int K, int d, float p, uint64_t seed
     if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
-    return launch_debug_masks(B, T, K, d, mk, (uint32_t)seq_base, out_bits, static_cast<cudaStream_t>(stream));
+    return launch_debug_masks(B, T, K, d, mk, (uint32_t)seq_base, c->mask_mode, out_bits, static_cast<cudaStream_t>(stream));
 }
 
 int dm_device_error(dm_ctx* c, void* stream, uint32_t* out_code) {

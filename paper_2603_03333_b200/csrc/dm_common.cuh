@@ -21,7 +21,7 @@ enum : uint32_t {
 struct RowKey {
     int q;        // hidden row index into H
     uint32_t s;   // sequence id (low 32 bits)
-    uint32_t t;   // position index within the sequence
+    uint32_t t;   // position index in the mask key (0 when masks are shared across positions)
     uint32_t i;   // path index
 };
 
@@ -32,6 +32,7 @@ struct RowMap {
     const int32_t* sel;
     int K, T, B;
     uint32_t seq_base_lo;
+    int shared_masks;   // 1: the mask key ignores the position (one mask per sequence and path)
 };
 
 __device__ __forceinline__ bool row_key(const RowMap& m, int r, RowKey& k) {
@@ -40,14 +41,14 @@ __device__ __forceinline__ bool row_key(const RowMap& m, int r, RowKey& k) {
         k.q = q;
         k.i = (uint32_t)(r - q * m.K);
         int b = q / m.T;
-        k.t = (uint32_t)(q - b * m.T);
+        k.t = m.shared_masks ? 0u : (uint32_t)(q - b * m.T);
         k.s = m.seq_base_lo + (uint32_t)b;
         return true;
     }
     int b = m.sel[3 * r], t = m.sel[3 * r + 1], i = m.sel[3 * r + 2];
     bool ok = b >= 0 && b < m.B && t >= 0 && t < m.T && i >= 0;
     k.q = ok ? b * m.T + t : 0;
-    k.t = (uint32_t)t;
+    k.t = m.shared_masks ? 0u : (uint32_t)t;
     k.i = (uint32_t)i;
     k.s = m.seq_base_lo + (uint32_t)b;
     return ok;

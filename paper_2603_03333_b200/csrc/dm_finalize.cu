@@ -28,13 +28,13 @@ int launch_finalize(const unsigned long long* partials, int n_slices, int rows,
 }
 
 // Eq. 1 keep bits, one 32-bit word (eight Philox quads) per thread.
-__global__ void debug_masks_kernel(int n_paths, int K, int T, int d, MaskKey mk, uint32_t seq_base_lo,
+__global__ void debug_masks_kernel(int n_paths, int K, int T, int d, MaskKey mk, uint32_t seq_base_lo, int shared_masks,
                                    uint32_t* __restrict__ out_bits) {
     const int words = (d + 31) / 32;
     const long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (x >= (long long)n_paths * words) return;
     const int r = (int)(x / words), w = (int)(x - (long long)r * words);
-    RowMap map{nullptr, K, T, 0, seq_base_lo};
+    RowMap map{nullptr, K, T, 0, seq_base_lo, shared_masks};
     RowKey k;
     row_key(map, r, k);
     uint32_t bits = 0;
@@ -49,14 +49,14 @@ __global__ void debug_masks_kernel(int n_paths, int K, int T, int d, MaskKey mk,
     out_bits[x] = bits;
 }
 
-int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo,
+int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo, int shared_masks,
                        uint32_t* out_bits, cudaStream_t stream) {
     const long long n_paths = (long long)B * T * K;
     const long long total = n_paths * ((d + 31) / 32);
     if (total > (1ll << 40)) return DM_EUNSUPPORTED;
     const long long blocks = (total + 255) / 256;
     if (blocks > 0x7FFFFFFFll) return DM_EUNSUPPORTED;
-    debug_masks_kernel<<<(unsigned)blocks, 256, 0, stream>>>((int)n_paths, K, T, d, mk, seq_base_lo, out_bits);
+    debug_masks_kernel<<<(unsigned)blocks, 256, 0, stream>>>((int)n_paths, K, T, d, mk, seq_base_lo, shared_masks, out_bits);
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 

@@ -72,7 +72,7 @@ int launch_js(const float* logits, const float* draft_prob, float* workspace, in
               const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
               int32_t* out_accept_len, cudaStream_t stream);
 
-int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo,
+int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo, int shared_masks,
                        uint32_t* out_bits, cudaStream_t stream);
 
 }  // namespace dm

@@ -208,3 +208,29 @@ def test_argument_errors(ctx):
     # the context still works after the refused calls
     ok = ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED)
     assert int(ok["accept_len"][0]) <= cfg.T
+
+
+def test_shared_mask_mode(ctx):
+    """DM_MASK_PER_PATH: masks, tokens, counts and accepted lengths against the oracle's shared-mask
+    reading; the masks of every position equal those of position 0."""
+    cfg = wl.Config("shared", d=256, V=3000, dtype=wl.BF16, B=2, T=4, K=8, p=0.3)
+    work = wl.make_workload(cfg, device=DEV)
+    ctx.set_head(work.W, max_rows=cfg.rows)
+    ctx.set_mask_mode(binding.MASK_PER_PATH)
+    try:
+        bits = ctx.debug_masks(cfg.B, cfg.T, cfg.K, cfg.d, cfg.p, SEED, seq_base=2).cpu().numpy().view(np.uint32)
+        ref_bits = oracle.masks(cfg.B, 1, cfg.K, cfg.d, cfg.p, SEED, 2)          # position 0 of each sequence
+        for t in range(cfg.T):
+            assert np.array_equal(bits[:, t], ref_bits[:, 0])
+        ref = oracle.verify_batched(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H),
+                                    work.draft.cpu().numpy(), cfg.K, cfg.p, SEED, seq_base=2, shared_masks=True)
+        for impl in _impls(ctx, cfg):
+            ctx.set_impl(impl)
+            got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=2))
+            ctx.set_impl(binding.IMPL_AUTO)
+            assert ctx.device_error() == 0
+            check_chain(got, ref, work.draft.cpu().numpy())
+    finally:
+        ctx.set_mask_mode(binding.MASK_PER_POSITION)
+    with pytest.raises(pk.DropMatchError):
+        ctx.set_mask_mode(7)

@@ -155,3 +155,25 @@ def test_nested_paths_make_acceptance_monotone_in_K():
         assert np.all(out["accept_len"] <= T)
         assert np.all(out["counts"].max(-1) <= K) and np.all(out["counts"] >= 1)
         prev = out
+
+
+def test_shared_masks_make_paths_persistent_heads():
+    """Other reading of Eq. 1 (no position index on m^(i)): with shared masks a path applies one
+    mask at every position, so equal hidden rows decode to equal tokens path by path, and the
+    tokens of position t equal those of a single-position call on that row (which has t = 0)."""
+    rng = np.random.default_rng(21)
+    V, d, T, K, p, seed = 200, 48, 4, 6, 0.4, 77
+    W = (rng.normal(size=(V, d)) * 0.4).astype(np.float32)
+    row = rng.normal(size=d).astype(np.float32)
+    H = np.tile(row, (1, T, 1))                                  # the same hidden row at every position
+    draft = np.zeros((1, T), dtype=np.int32)
+    sh = oracle.verify_batched(W, oracle.F32, H, draft, K, p, seed, seq_base=5, shared_masks=True)
+    ind = oracle.verify_batched(W, oracle.F32, H, draft, K, p, seed, seq_base=5)
+    assert (sh["tokens"] == sh["tokens"][:, :1]).all()           # identical across positions, path by path
+    assert not (ind["tokens"] == ind["tokens"][:, :1]).all()     # independent masks: they differ somewhere
+    assert np.array_equal(sh["tokens"][0, 0], ind["tokens"][0, 0])   # position 0 is keyed alike in both readings
+    H2 = rng.normal(size=(1, T, d)).astype(np.float32)
+    sh2 = oracle.verify_batched(W, oracle.F32, H2, draft, K, p, seed, seq_base=5, shared_masks=True)
+    for t in range(T):                                           # position t under shared masks == that row alone
+        one = oracle.verify_batched(W, oracle.F32, H2[:, t:t + 1], draft[:, :1], K, p, seed, seq_base=5)
+        assert np.array_equal(sh2["tokens"][0, t], one["tokens"][0, 0])
