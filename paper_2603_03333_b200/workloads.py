@@ -49,6 +49,8 @@ CONFIGS = {
     "qwen8b": Config("qwen8b", d=4096, V=151936, dtype=BF16, B=1, T=7, K=8, p=0.1),
     "tree": Config("tree", d=4096, V=128256, dtype=BF16, B=4, T=61, K=8, p=0.1, kind="tree", N=60),
     "llama70b": Config("llama70b", d=8192, V=128256, dtype=BF16, B=16, T=8, K=16, p=0.1),
+    # the Llama-3-8B head at the upper end of the HBM-bound range (256 paths: staged operand, CTA pairs)
+    "llama8b_k32": Config("llama8b_k32", d=4096, V=128256, dtype=BF16, B=1, T=8, K=32, p=0.1),
 }
 
 
