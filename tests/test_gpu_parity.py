@@ -234,3 +234,38 @@ def test_shared_mask_mode(ctx):
         ctx.set_mask_mode(binding.MASK_PER_POSITION)
     with pytest.raises(pk.DropMatchError):
         ctx.set_mask_mode(7)
+
+
+EDGE = [
+    # one position whose 300 paths straddle two launches of the tensor-core kernel
+    wl.Config("edge_k300", d=128, V=2000, dtype=wl.BF16, B=1, T=1, K=300, p=0.2),
+    # almost everything dropped: many all-zero masked rows, all-zero logits, ties resolved to token 0
+    wl.Config("edge_p_high", d=64, V=300, dtype=wl.BF16, B=2, T=3, K=16, p=0.97),
+    # a one-word vocabulary and a two-word one
+    wl.Config("edge_v1", d=64, V=1, dtype=wl.BF16, B=1, T=2, K=4, p=0.1, draft_mode="toy"),
+    wl.Config("edge_v2", d=128, V=2, dtype=wl.BF16, B=1, T=3, K=8, p=0.5, draft_mode="toy"),
+    # widest single launch exactly (256 paths) and one more (257)
+    wl.Config("edge_rows256", d=64, V=40000, dtype=wl.BF16, B=1, T=8, K=32, p=0.1),
+    wl.Config("edge_rows257", d=64, V=1000, dtype=wl.BF16, B=1, T=1, K=257, p=0.1),
+    # fp32 head whose hidden size is the minimum the CUDA-core kernel takes
+    wl.Config("edge_f32_d4", d=4, V=50, dtype=wl.F32, B=1, T=2, K=16, p=0.5, draft_mode="toy"),
+]
+
+
+@pytest.mark.parametrize("cfg", EDGE, ids=lambda c: c.name)
+def test_edge_shapes(ctx, cfg):
+    if cfg.V < 5:   # the workload recipe draws drafts from a top-5: build the few inputs by hand
+        W = wl.make_head(cfg.V, cfg.d, cfg.dtype, seed=1, device=DEV)
+        H = wl.make_hidden(cfg.B * cfg.T, cfg.d, cfg.dtype, seed=2, device=DEV).view(cfg.B, cfg.T, cfg.d)
+        draft = torch.zeros((cfg.B, cfg.T), dtype=torch.int32, device=DEV)
+        work = wl.Workload(cfg, W, H, draft, None, None, None)
+    else:
+        work = wl.make_workload(cfg, device=DEV)
+    for impl in _impls(ctx, cfg):
+        got, ref, n_diff, _ = _run_chain(ctx, cfg, impl, work=work)
+        assert n_diff <= max(2, cfg.rows // 10)
+    if cfg.name == "edge_p_high":
+        zero_rows = (oracle.masks(cfg.B, cfg.T, cfg.K, cfg.d, cfg.p, SEED, 0) == 0).all(axis=-1)
+        assert zero_rows.any()                                   # some paths really dropped everything ...
+        assert (ref["tokens"][zero_rows] == 0).all()             # ... and decode to token 0 on both sides
+        assert (got["tokens"][zero_rows] == 0).all()
