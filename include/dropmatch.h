@@ -108,6 +108,24 @@ int dropmatch_verify_batched(dm_ctx* ctx, const void* H, const int32_t* draft, i
                              int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
                              int32_t* out_accept_len, void* stream);
 
+/* dropmatch_verify_batched plus the token the engine emits after the accepted prefix.  Every
+ * hidden row gets, in the same pass over W, one more path without dropout: the target model's own
+ * greedy token (the paper does not say how DropMatch picks the correction or bonus token; this
+ * is the choice of plain speculative decoding with greedy verification).
+ *   H[B, T + bonus_row, d]   bonus_row = 1: one more hidden row per sequence, the state after the
+ *                            last draft token, so that a fully accepted draft yields a bonus token
+ *   draft[B,T]               as before; positions 0..T-1 are scanned
+ *   out_tokens, out_counts   [B, T + bonus_row, K] (the extra row's paths are computed too)
+ *   out_draft_hits           [B,T] or NULL
+ *   out_plain_tokens         [B, T + bonus_row]: argmax of the undropped head per hidden row
+ *   out_next_token[B]        out_plain_tokens[b, accept_len[b]], or -1 if that row does not exist
+ * Counts B*(T+bonus_row)*(K+1) rows against max_rows of dm_set_head.  K <= 1023. */
+int dropmatch_verify_batched_next(dm_ctx* ctx, const void* H, const int32_t* draft, int B, int T, int bonus_row,
+                                  int K, float p, uint64_t seed, uint64_t seq_base, int rule,
+                                  int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
+                                  int32_t* out_accept_len, int32_t* out_plain_tokens, int32_t* out_next_token,
+                                  void* stream);
+
 /* Same as dropmatch_verify_batched, but H, draft and all outputs are HOST pointers (pinned or
  * pageable).  Gathers the inputs in the context's pinned buffer and sends them with one copy,
  * runs the call with its outputs going to pinned memory the device can write, waits for

@@ -78,6 +78,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_verify_tree.argtypes = [vp, ci, ci, ci, vp, i32p, i32p, i32p, ci, ci, ci, ci, cf,
                                          u64, u64, ci, i32p, f64p, i32p, i32p, i32p, i32p]
         L.oracle_verify_tree.restype = None
+        L.oracle_verify_batched_next.argtypes = [vp, ci, ci, ci, vp, i32p, ci, ci, ci, ci, cf, u64, u64, ci,
+                                                 i32p, f64p, i32p, i32p, i32p, i32p, f64p, i32p]
+        L.oracle_verify_batched_next.restype = None
         L.oracle_js_divergence.argtypes = [f64p, f64p, ci]
         L.oracle_js_divergence.restype = ctypes.c_double
         L.oracle_js_from_logits.argtypes = [f64p, ci, ci, f64p, f64p]
@@ -297,3 +300,30 @@ def verify_js(W, dtype, H, draft, draft_prob, K, p, seed, seq_base=0):
                            seq_base, tokens.ctypes.data_as(i32p), cnt.ctypes.data_as(i32p), _f64p(js),
                            js_ok.ctypes.data_as(i32p), alen.ctypes.data_as(i32p))
     return dict(tokens=tokens, counts=cnt, js=js, js_ok=js_ok, accept_len=alen)
+
+
+def verify_batched_next(W, dtype, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE):
+    """H[B,T_h,d] with T_h = T or T+1, draft[B,T] -> verify_batched's outputs (tokens/counts over
+    T_h rows) plus plain[B,T_h], plain_gap, next[B]."""
+    Ws, Hs = _store(W, dtype), _store(H, dtype)
+    V, d = Ws.shape
+    B, T_h, d2 = Hs.shape
+    dr, drp = _i32(draft)
+    T = dr.shape[1]
+    assert d2 == d and dr.shape[0] == B and T_h - T in (0, 1)
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    tokens = np.zeros((B, T_h, K), dtype=np.int32)
+    gap = np.zeros((B, T_h, K), dtype=np.float64)
+    cnt = np.zeros((B, T_h, K), dtype=np.int32)
+    hits = np.zeros((B, T), dtype=np.int32)
+    alen = np.zeros((B,), dtype=np.int32)
+    plain = np.zeros((B, T_h), dtype=np.int32)
+    pgap = np.zeros((B, T_h), dtype=np.float64)
+    nxt = np.zeros((B,), dtype=np.int32)
+    lib().oracle_verify_batched_next(Ws.ctypes.data, dtype, V, d, Hs.ctypes.data, drp, B, T, T_h - T, K,
+                                     float(np.float32(p)), seed, seq_base, rule, tokens.ctypes.data_as(i32p),
+                                     _f64p(gap), cnt.ctypes.data_as(i32p), hits.ctypes.data_as(i32p),
+                                     alen.ctypes.data_as(i32p), plain.ctypes.data_as(i32p), _f64p(pgap),
+                                     nxt.ctypes.data_as(i32p))
+    return dict(tokens=tokens, gap=gap, counts=cnt, hits=hits, accept_len=alen, plain=plain, plain_gap=pgap,
+                next=nxt)

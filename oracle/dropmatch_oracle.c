@@ -434,3 +434,52 @@ void oracle_verify_js(const void *W, int dtype, int V, int d, const void *H, con
     free(logits);
     free(dp);
 }
+
+/* ------------------------------------------------------------------------- */
+/* Token emitted after the accepted prefix                                    */
+/* ------------------------------------------------------------------------- */
+
+/* Chain verification as oracle_verify_batched, on H[B, T_h, d] with T_h = T + bonus_row hidden
+ * rows per sequence (only the first T are scanned against draft[B,T]), plus the target's own
+ * greedy token of every hidden row, plain[b,q] = argmax_v (W h_{b,q})[v] (no dropout), and
+ * next[b] = plain[b, accept_len[b]] if that row exists, else -1.  The paper leaves the choice of
+ * this token open; this is greedy verification's.  plain_gap may be NULL. */
+void oracle_verify_batched_next(const void *W, int dtype, int V, int d, const void *H,
+                                const int32_t *draft, int B, int T, int bonus_row, int K, float p,
+                                uint64_t seed, uint64_t seq_base, int rule, int32_t *out_tokens,
+                                double *out_gap, int32_t *out_counts, int32_t *out_hits,
+                                int32_t *out_accept_len, int32_t *out_plain, double *plain_gap,
+                                int32_t *out_next)
+{
+    const int T_h = T + (bonus_row ? 1 : 0);
+    const size_t elem = (dtype == ORACLE_F32) ? 4 : 2;
+    sample_tokens(W, dtype, V, d, H, B * T_h, T_h, K, p, seed, seq_base, 0, out_tokens, out_gap);
+    double *logits = (double *)malloc((size_t)V * sizeof(double));
+    for (int b = 0; b < B; ++b) {
+        for (int q = 0; q < T_h; ++q) {
+            const size_t row = (size_t)b * T_h + q;
+            const char *h_row = (const char *)H + row * d * elem;
+#pragma omp parallel for schedule(static)
+            for (int v = 0; v < V; ++v) {
+                double acc = 0.0;
+                for (int j = 0; j < d; ++j)
+                    acc += load_elem(W, dtype, (size_t)v * d + j) * load_elem(h_row, dtype, (size_t)j);
+                logits[v] = acc;
+            }
+            double gap;
+            out_plain[row] = oracle_argmax(logits, V, &gap);
+            if (plain_gap) plain_gap[row] = gap;
+            int hits = oracle_counts(out_tokens + row * K, K, q < T ? draft[(size_t)b * T + q] : -1,
+                                     out_counts + row * K);
+            if (out_hits && q < T) out_hits[(size_t)b * T + q] = hits;
+        }
+        /* scan the T draft positions; the token rows of a sequence are T_h apart */
+        int len = 0;
+        while (len < T && oracle_position_ok(out_tokens + ((size_t)b * T_h + len) * K, K,
+                                             draft[(size_t)b * T + len], rule))
+            ++len;
+        out_accept_len[b] = len;
+        out_next[b] = (len < T_h) ? out_plain[(size_t)b * T_h + len] : -1;
+    }
+    free(logits);
+}

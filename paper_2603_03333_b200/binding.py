@@ -32,6 +32,8 @@ SIGNATURES = {
     "dm_set_mask_mode": (_ci, [_vp, _ci]),
     "dropmatch_verify": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _u64, _ci, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_batched_next": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
+                                            _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_static": (_ci, [_ci, _vp, _ci, _ci, _ci, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
                                               _vp, _vp, _vp, _vp, _vp]),
@@ -175,6 +177,24 @@ class Context:
                                               _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["hits"]),
                                               _ptr(out["accept_len"]), _stream(self.device)),
                "dropmatch_verify_batched")
+        return out
+
+    # -- dropmatch_verify_batched_next
+    def verify_batched_next(self, H, draft, K, p, seed, seq_base=0, rule=RULE_NAIVE):
+        """H[B,T_h,d] with T_h = T or T+1 (bonus row), draft[B,T].  Adds plain[B,T_h], next[B]."""
+        B, T_h, _ = H.shape
+        T = draft.shape[1]
+        if T_h - T not in (0, 1):
+            raise TypeError("H must have T or T+1 hidden rows per sequence")
+        _dev(H, self._tdtype(), "H"); _dev(draft, torch.int32, "draft")
+        i32 = dict(dtype=torch.int32, device=self.device)
+        out = dict(tokens=torch.empty((B, T_h, K), **i32), counts=torch.empty((B, T_h, K), **i32),
+                   hits=torch.empty((B, T), **i32), accept_len=torch.empty((B,), **i32),
+                   plain=torch.empty((B, T_h), **i32), next=torch.empty((B,), **i32))
+        _check(lib().dropmatch_verify_batched_next(self._h, _ptr(H), _ptr(draft), B, T, T_h - T, K, p, seed, seq_base,
+                                                   rule, _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["hits"]),
+                                                   _ptr(out["accept_len"]), _ptr(out["plain"]), _ptr(out["next"]),
+                                                   _stream(self.device)), "dropmatch_verify_batched_next")
         return out
 
     def alloc_outputs(self, B, T, K):

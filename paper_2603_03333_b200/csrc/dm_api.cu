@@ -97,7 +97,7 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
                const FinalizeArgs& fa, cudaStream_t stream, float* logits_out = nullptr) {
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
     if (rows > c->max_rows) return DM_EWORKSPACE;
-    if (finalize_smem_bytes(fa.T, fa.K, fa.N) > 200 * 1024) return DM_EUNSUPPORTED;
+    if (finalize_smem_bytes(fa.T, fa.K + fa.plain, fa.N) > 200 * 1024) return DM_EUNSUPPORTED;
     int impl;
     int st = pick_impl(c, rows, &impl);
     if (st != DM_OK) return st;
@@ -263,6 +263,36 @@ int dropmatch_verify_batched(dm_ctx* c, const void* H, const int32_t* draft, int
     fa.N = 0;
     fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
     return run_verify(c, H, B * T * K, map, mk, fa, static_cast<cudaStream_t>(stream));
+}
+
+int dropmatch_verify_batched_next(dm_ctx* c, const void* H, const int32_t* draft, int B, int T, int bonus_row,
+                                  int K, float p, uint64_t seed, uint64_t seq_base, int rule,
+                                  int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
+                                  int32_t* out_accept_len, int32_t* out_plain_tokens, int32_t* out_next_token,
+                                  void* stream) {
+    if (bonus_row != 0 && bonus_row != 1) return DM_EINVAL;
+    const int T_h = T + bonus_row;   // hidden rows per sequence
+    int st = check_common(c, H, B, T_h, K);
+    if (st != DM_OK) return st;
+    if (T < 1 || K + 1 > kMaxK) return DM_EINVAL;
+    if (draft == nullptr || out_tokens == nullptr || out_counts == nullptr || out_accept_len == nullptr ||
+        out_plain_tokens == nullptr || out_next_token == nullptr)
+        return DM_EINVAL;
+    if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
+    if ((long long)B * T_h * (K + 1) > 0x3FFFFFFFll) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    RowMap map{nullptr, K, T_h, B, (uint32_t)seq_base, c->mask_mode, 1};
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = T_h; fa.K = K; fa.rule = rule;
+    fa.plain = 1; fa.T_draft = T;
+    fa.out_plain = out_plain_tokens; fa.out_next = out_next_token;
+    fa.draft = draft; fa.out_hits = out_draft_hits;
+    fa.N = 0;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    return run_verify(c, H, B * T_h * (K + 1), map, mk, fa, static_cast<cudaStream_t>(stream));
 }
 
 int dropmatch_verify(dm_ctx* c, const void* H, const int32_t* draft, int T, int K, float p,

@@ -33,13 +33,17 @@ struct RowMap {
     int K, T, B;
     uint32_t seq_base_lo;
     int shared_masks;   // 1: the mask key ignores the position (one mask per sequence and path)
+    int plain_extra;    // 1: K+1 paths per hidden row, the last one unmasked (path index kPlainPath)
 };
+constexpr uint32_t kPlainPath = 0xFFFFFFFFu;   // RowKey.i of a path that keeps every element
 
 __device__ __forceinline__ bool row_key(const RowMap& m, int r, RowKey& k) {
     if (m.sel == nullptr) {
-        int q = r / m.K;
+        const int kp = m.K + m.plain_extra;
+        int q = r / kp;
         k.q = q;
-        k.i = (uint32_t)(r - q * m.K);
+        k.i = (uint32_t)(r - q * kp);
+        if (m.plain_extra && k.i == (uint32_t)m.K) k.i = kPlainPath;
         int b = q / m.T;
         k.t = m.shared_masks ? 0u : (uint32_t)(q - b * m.T);
         k.s = m.seq_base_lo + (uint32_t)b;
@@ -74,6 +78,7 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
 // Keep flags (bit n = element 4*quad + n kept) of one Philox quad of a path.
 __device__ __forceinline__ uint32_t keep4(uint32_t quad, const RowKey& k, uint32_t key0,
                                           uint32_t key1, uint32_t thr) {
+    if (k.i == kPlainPath) return 0xFu;   // the unmasked path of a hidden row
     uint4 w = philox4x32_10(make_uint4(quad, k.i, k.t, k.s), key0, key1);
     return (w.x >= thr ? 1u : 0u) | (w.y >= thr ? 2u : 0u) | (w.z >= thr ? 4u : 0u) |
            (w.w >= thr ? 8u : 0u);

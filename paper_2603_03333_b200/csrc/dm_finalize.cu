@@ -18,7 +18,7 @@ size_t finalize_smem_bytes(int T, int K, int N) {
 
 int launch_finalize(const unsigned long long* partials, int n_slices, int rows,
                     const FinalizeArgs& a, cudaStream_t stream) {
-    const size_t smem = finalize_smem_bytes(a.T, a.K, a.N);
+    const size_t smem = finalize_smem_bytes(a.T, a.K + a.plain, a.N);   // the scratch keeps the unmasked path too
     if (smem > 200 * 1024) return DM_EUNSUPPORTED;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

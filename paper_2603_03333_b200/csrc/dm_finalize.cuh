@@ -43,10 +43,21 @@ template <class Sync>
 __device__ __forceinline__ void finalize_sequence(const unsigned long long* partials, int n_slices, int rows,
                                                   const FinalizeArgs& a, int b, int32_t* sm, int tid,
                                                   int nthreads, Sync sync) {
-    const int TK = a.T * a.K;
-    int32_t* toks = sm;            // [T*K]
+    // Kp paths per hidden row: the K dropout paths and, if a.plain, one unmasked path after them
+    // (the target's own greedy token).  Outputs are compact [T][K]; the scratch keeps [T][Kp].
+    const int Kp = a.K + a.plain;
+    const int Td = a.T_draft > 0 ? a.T_draft : a.T;   // draft positions that are scanned (<= T)
+    const int TK = a.T * Kp;
+    int32_t* toks = sm;            // [T*Kp]
     int32_t* flag = sm + TK;       // chain: ok[T]; tree: test[N] then ok/depth packed [N]
     const size_t row0 = (size_t)b * TK;
+    const size_t out0 = (size_t)b * a.T * a.K;
+    auto store_token = [&](int x, int32_t tok) {
+        toks[x] = tok;
+        const int t = x / Kp, i = x - t * Kp;
+        if (i < a.K) a.out_tokens[out0 + (size_t)t * a.K + i] = tok;
+        else if (a.out_plain) a.out_plain[(size_t)b * a.T + t] = tok;
+    };
 
     // split-V merge: the packed (key, inverted index) maximum over slices is the argmax with
     // the smallest index on ties.  Many slices: one warp per row, lanes stride over the slices.
@@ -60,9 +71,7 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
                 unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x);
                 best = c > best ? c : best;
             }
-            int32_t tok = (int32_t)best_index(best);
-            toks[x] = tok;
-            a.out_tokens[row0 + x] = tok;
+            store_token(x, (int32_t)best_index(best));
         }
     } else {
         for (int x0 = warp * 4; x0 < TK; x0 += n_warps * 4) {   // four rows at a time: their loads overlap
@@ -83,37 +92,37 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
                     unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best[u], off);
                     best[u] = o > best[u] ? o : best[u];
                 }
-                if (lane == 0 && x0 + u < TK) {
-                    int32_t tok = (int32_t)best_index(best[u]);
-                    toks[x0 + u] = tok;
-                    a.out_tokens[row0 + x0 + u] = tok;
-                }
+                if (lane == 0 && x0 + u < TK) store_token(x0 + u, (int32_t)best_index(best[u]));
             }
         }
     }
     sync();
 
     // empirical distribution: multiplicity of every sampled token within its position
-    for (int x = tid; x < TK; x += nthreads) {
-        const int32_t* row = toks + (x / a.K) * a.K;
-        int32_t y = toks[x];
+    for (int x = tid; x < a.T * a.K; x += nthreads) {
+        const int t = x / a.K;
+        const int32_t* row = toks + t * Kp;
+        int32_t y = row[x - t * a.K];
         int c = 0;
         for (int i = 0; i < a.K; ++i) c += (row[i] == y);
-        a.out_counts[row0 + x] = c;
+        a.out_counts[out0 + x] = c;
     }
 
     if (a.N == 0) {
-        for (int t = tid; t < a.T; t += nthreads) {
+        for (int t = tid; t < Td; t += nthreads) {
             int hits;
-            bool ok = position_ok(toks + t * a.K, a.K, a.draft[(size_t)b * a.T + t], a.rule, &hits);
+            bool ok = position_ok(toks + t * Kp, a.K, a.draft[(size_t)b * Td + t], a.rule, &hits);
             flag[t] = ok;
-            if (a.out_hits) a.out_hits[(size_t)b * a.T + t] = hits;
+            if (a.out_hits) a.out_hits[(size_t)b * Td + t] = hits;
         }
         sync();
         if (tid == 0) {
             int len = 0;
-            while (len < a.T && flag[len]) ++len;   // first rejection ends acceptance
+            while (len < Td && flag[len]) ++len;   // first rejection ends acceptance
             a.out_accept_len[b] = len;
+            // the token the engine emits next: the target's greedy token at the first position
+            // that was not accepted (a correction), or after all of them if that row was given
+            if (a.out_next) a.out_next[b] = (a.plain && len < a.T) ? toks[len * Kp + a.K] : -1;
         }
         sync();   // the scratch may be reused for the next sequence
         return;
@@ -125,7 +134,7 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
     for (int n = tid; n < a.N; n += nthreads) {
         int h = a.node_hrow[n0 + n];
         bool ok = false;
-        if (h >= 0 && h < a.T) ok = position_ok(toks + h * a.K, a.K, a.node_token[n0 + n], a.rule, nullptr);
+        if (h >= 0 && h < a.T) ok = position_ok(toks + h * Kp, a.K, a.node_token[n0 + n], a.rule, nullptr);
         flag[n] = ok;
         depth[n] = a.node_parent[n0 + n];   // staged here so that the serial walk stays in shared memory
     }

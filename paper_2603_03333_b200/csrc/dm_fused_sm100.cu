@@ -791,7 +791,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.partials = partials; P.dbg_logits = dbg_logits; P.err = err;
         // a call of one launch finishes itself; larger calls leave it to finalize_kernel
         P.fold = (fin != nullptr && ticket != nullptr && best != nullptr && rows <= kMaxNPad &&
-                  finalize_smem_bytes(fin->T, fin->K, fin->N) <= 32 * 1024) ? 1 : 0;
+                  finalize_smem_bytes(fin->T, fin->K + fin->plain, fin->N) <= 32 * 1024) ? 1 : 0;
         P.ticket = ticket;
         P.best = best;
         if (P.fold) { P.fin = *fin; if (folded_out) *folded_out = true; }

@@ -28,7 +28,11 @@ struct MaskKey {
 
 // Acceptance inputs/outputs handed to the finalize kernel.
 struct FinalizeArgs {
-    int B, T, K, rule;
+    int B, T, K, rule;     // T hidden rows per sequence, K dropout paths per row
+    int plain;             // 1: every hidden row has one more, unmasked path after its K dropout paths
+    int T_draft;           // draft positions scanned per sequence (0 = T); T - T_draft extra hidden rows
+    int32_t* out_plain;    // [B,T] token of the unmasked path, or null
+    int32_t* out_next;     // [B] unmasked token at position accept_len (-1 if there is no such row), or null
     // chain
     const int32_t* draft;        // [B,T] or null (tree)
     int32_t* out_hits;           // [B,T] or null

@@ -269,3 +269,40 @@ def test_edge_shapes(ctx, cfg):
         assert zero_rows.any()                                   # some paths really dropped everything ...
         assert (ref["tokens"][zero_rows] == 0).all()             # ... and decode to token 0 on both sides
         assert (got["tokens"][zero_rows] == 0).all()
+
+
+@pytest.mark.parametrize("bonus", [0, 1])
+@pytest.mark.parametrize("cfg", [
+    wl.Config("next_bf16", d=256, V=3000, dtype=wl.BF16, B=3, T=4, K=8, p=0.2),          # one launch, finished in-kernel
+    wl.Config("next_bf16_wide", d=128, V=60000, dtype=wl.BF16, B=2, T=5, K=31, p=0.1),   # staged, several launches
+    wl.Config("next_f32", d=100, V=517, dtype=wl.F32, B=2, T=3, K=7, p=0.2, draft_mode="toy"),
+], ids=lambda c: c.name)
+def test_next_token_call(ctx, cfg, bonus):
+    T_h = cfg.T + bonus
+    work = wl.make_workload(cfg.with_(T=T_h), device=DEV)              # T_h hidden rows; drafts for the first T
+    draft = work.draft[:, :cfg.T].contiguous()
+    ctx.set_head(work.W, max_rows=cfg.B * T_h * (cfg.K + 1))
+    ref = oracle.verify_batched_next(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H),
+                                     draft.cpu().numpy(), cfg.K, cfg.p, SEED, seq_base=4)
+    for impl in _impls(ctx, cfg):
+        ctx.set_impl(impl)
+        got = to_np(ctx.verify_batched_next(work.H, draft, cfg.K, cfg.p, SEED, seq_base=4))
+        ctx.set_impl(binding.IMPL_AUTO)
+        assert ctx.device_error() == 0
+        bad = (got["tokens"] != ref["tokens"]) & (ref["gap"] >= NEAR_TIE)
+        assert not bad.any()
+        bad_plain = (got["plain"] != ref["plain"]) & (ref["plain_gap"] >= NEAR_TIE)
+        assert not bad_plain.any()
+        d_np = draft.cpu().numpy()
+        for b in range(cfg.B):                                          # integer stages from the GPU's own tokens
+            n = oracle.accept_chain(got["tokens"][b, :cfg.T], d_np[b], oracle.RULE_NAIVE)
+            assert got["accept_len"][b] == n
+            assert got["next"][b] == (got["plain"][b, n] if n < T_h else -1)
+            for t in range(T_h):
+                cnt, hits = oracle.counts(got["tokens"][b, t], int(d_np[b, t]) if t < cfg.T else -1)
+                assert np.array_equal(got["counts"][b, t], cnt)
+                if t < cfg.T:
+                    assert got["hits"][b, t] == hits
+        if not (got["tokens"] != ref["tokens"]).any() and not (got["plain"] != ref["plain"]).any():
+            for key in ("counts", "hits", "accept_len", "next"):
+                assert np.array_equal(got[key], ref[key]), key

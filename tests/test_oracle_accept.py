@@ -177,3 +177,36 @@ def test_shared_masks_make_paths_persistent_heads():
     for t in range(T):                                           # position t under shared masks == that row alone
         one = oracle.verify_batched(W, oracle.F32, H2[:, t:t + 1], draft[:, :1], K, p, seed, seq_base=5)
         assert np.array_equal(sh2["tokens"][0, t], one["tokens"][0, 0])
+
+
+@pytest.mark.parametrize("bonus", [0, 1])
+def test_next_token_is_the_plain_greedy_token_at_the_first_unaccepted_position(bonus):
+    """Pins for oracle.verify_batched_next: the plain tokens are a library fp64 GEMV argmax; the
+    dropout part equals verify_batched on the same rows; next[b] follows from a brute-force scan."""
+    rng = np.random.default_rng(31 + bonus)
+    V, d, B, T, K, p, seed = 150, 40, 3, 4, 5, 0.3, 1234
+    T_h = T + bonus
+    W = (rng.normal(size=(V, d)) * 0.5).astype(np.float32)
+    H = rng.normal(size=(B, T_h, d)).astype(np.float32)
+    und = np.einsum("bqd,vd->bqv", H.astype(np.float64), W.astype(np.float64))
+    greedy = und.argmax(-1).astype(np.int32)
+    draft = greedy[:, :T].copy()
+    draft[0, 2] = (draft[0, 2] + 1) % V            # sequence 0: a wrong draft at position 2
+    draft[1, 0] = (draft[1, 0] + 1) % V            # sequence 1: wrong at once; sequence 2: all plausible
+    out = oracle.verify_batched_next(W, oracle.F32, H, draft, K, p, seed, seq_base=9)
+    assert np.array_equal(out["plain"], greedy)
+    if bonus == 0:                                  # same rows, same keys: the dropout part is the plain call's
+        ref = oracle.verify_batched(W, oracle.F32, H, draft, K, p, seed, seq_base=9)
+        for key in ("tokens", "counts", "hits", "accept_len"):
+            assert np.array_equal(out[key], ref[key]), key
+    for b in range(B):
+        n = 0
+        while n < T and draft[b, n] in out["tokens"][b, n]:
+            n += 1
+        assert out["accept_len"][b] == n
+        assert out["next"][b] == (greedy[b, n] if n < T_h else -1)
+    # p = 0: every dropout path is the plain token, everything plausible is accepted
+    out0 = oracle.verify_batched_next(W, oracle.F32, H, greedy[:, :T].copy(), K, 0.0, seed)
+    assert (out0["tokens"] == out0["plain"][..., None]).all()
+    assert (out0["accept_len"] == T).all()
+    assert np.array_equal(out0["next"], greedy[:, T] if bonus else np.full(B, -1))
