@@ -70,10 +70,11 @@ struct FusedParams {
     int n_slots;      // accumulator slots in TMEM (512 / n_pad)
     int nsw, nsb;     // stages of the W ring and of the operand ring
     int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
+    int row_blocks;   // 1, or 2: two blocks of 256 paths share one pass over W (see fused_launch)
     RowMap map;
     uint32_t key0, key1, thr;
     float scale;
-    unsigned long long* partials;   // [gridDim.x][rows_total]
+    unsigned long long* partials;   // [vocabulary slice][rows_total]
     float* dbg_logits;              // [rows_total][V] or null
     uint32_t* err;
     // When `fold` is set the last CTA to finish also merges the partials and runs the histogram
@@ -125,6 +126,13 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int wps = kExpWarps / P.nsb;   // operand-builder warps per ring stage
     const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;   // 0 = leader of the pair
     const uint32_t dealloc_bar = slot_empty + 8 * P.n_slots;      // pair only: the other CTA is done with TMEM
+    // CTA -> (vocabulary slice, row block).  With two row blocks per launch the CTAs (or CTA pairs)
+    // alternate between the blocks: the two that share a slice run side by side and the second
+    // one's W loads hit L2, so that W crosses the HBM interface once for 512 paths.
+    const int unit = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // CTA, or CTA pair
+    const int rb = unit % P.row_blocks;
+    const int slice = kPair ? (unit / P.row_blocks) * 2 + (int)(blockIdx.x & 1) : unit / P.row_blocks;
+    const int row0 = P.row0 + rb * kMaxNPad;     // first path of this CTA's row block within the call
 
     if (threadIdx.x == 0) {
         ptx::prefetch_tensormap(&tmap_w);
@@ -151,7 +159,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     }
     for (int r = threadIdx.x; r < P.rows; r += kThreads) {
         RowKey k;
-        bool ok = row_key(P.map, P.row0 + r, k);
+        bool ok = row_key(P.map, row0 + r, k);
         if (!ok) atomicExch(P.err, (uint32_t)ERR_BAD_ROW);
         s_row[r] = RowInfo{ok ? k.q : -1, k.s, k.t, k.i};
     }
@@ -161,7 +169,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     ptx::tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
 
-    const int v_cta0 = blockIdx.x * P.slice_rows;
+    const int v_cta0 = slice * P.slice_rows;
     int my_tiles = 0;
     if (v_cta0 < P.V) {
         my_tiles = (P.V - v_cta0 + P.tile_rows - 1) / P.tile_rows;
@@ -278,7 +286,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             // thread streams the [n_pad x 64] block of every (group, block) step through TMA.
             if (threadIdx.x != (kFirstExpWarp + 4) * 32) return;
             const int b_rows = kPair ? P.n_pad / 2 : P.n_pad;      // a pair splits the operand rows
-            const int b_row0 = P.row0 + (int)rank * b_rows;
+            const int b_row0 = row0 + (int)rank * b_rows;
             const uint32_t b_stage_bytes = (uint32_t)b_rows * (kBlockK * 2);
             uint32_t bar_r = b_ready, bar_e = b_empty, dst = smem_base + P.off_b, parity = 1;
             int stage = 0;
@@ -435,7 +443,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
                             if (n0 + j < P.rows)
-                                P.dbg_logits[(size_t)(P.row0 + n0 + j) * P.V + v] =
+                                P.dbg_logits[(size_t)(row0 + n0 + j) * P.V + v] =
                                     s_row[n0 + j].q >= 0 ? __uint_as_float(acc[j]) * P.scale
                                                          : __uint_as_float(0x7FC00000u);
                     }
@@ -510,8 +518,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                 unsigned long long c = s_best[w * P.n_pad + n];
                 b = c > b ? c : b;
             }
-            if (P.fold) atomicMax(P.best + P.row0 + n, b);
-            else P.partials[(size_t)blockIdx.x * P.rows_total + P.row0 + n] = b;
+            if (P.fold) atomicMax(P.best + row0 + n, b);
+            else P.partials[(size_t)slice * P.rows_total + row0 + n] = b;
         }
         // ------------------------------------------------------------------ teardown
         // Every accumulator has been read, hence every MMA and every TMA load has completed.
@@ -580,9 +588,16 @@ mask_operand_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat16* __restri
 
 // ------------------------------------------------------------------------------ host side
 
+// How the vocabulary is cut for launches that cover `row_blocks` blocks of 256 paths at once:
+// the SMs are shared out between the row blocks, so a slice is `row_blocks` times longer.
+struct SliceGeometry {
+    CUtensorMap tmap_w;     // box [64 x tile_rows]
+    int n_ctas;             // CTAs per row block = vocabulary slices
+    int tiles_per_cta, tile_rows, slice_rows;
+};
+
 struct FusedState {
-    CUtensorMap tmap_w;
-    int n_ctas, tiles_per_cta, tile_rows, slice_rows;
+    SliceGeometry geo[2];   // [0]: one row block per launch, [1]: two
     // staging buffer for the masked operand of calls with too many rows for the in-kernel
     // builders, and one tensor map per box height n_pad = 16, 32, ..., 256 over it
     __nv_bfloat16* staging;
@@ -693,23 +708,30 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
         return DM_ECUDA;
     FusedState* fs = new (std::nothrow) FusedState();
     if (fs == nullptr) return DM_ECUDA;
-    int per = (head.V + sms - 1) / sms;
-    if (per < 64) per = 64;
-    fs->tiles_per_cta = (per + kTileM - 1) / kTileM;
-    fs->tile_rows = (per + fs->tiles_per_cta - 1) / fs->tiles_per_cta;
-    fs->slice_rows = fs->tiles_per_cta * fs->tile_rows;
-    fs->n_ctas = (head.V + fs->slice_rows - 1) / fs->slice_rows;
-
     EncodeTiledFn encode = encode_tiled_fn();
     if (encode == nullptr) { delete fs; return DM_ECUDA; }
     const cuuint64_t gdim[2] = {(cuuint64_t)head.d, (cuuint64_t)head.V};
     const cuuint64_t gstride[1] = {(cuuint64_t)head.d * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)fs->tile_rows};
     const cuuint32_t estride[2] = {1, 1};
-    CUresult r = encode(&fs->tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(head.W), gdim,
-                        gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { delete fs; return DM_ECUDA; }
+    CUresult r = CUDA_SUCCESS;
+    for (int g = 0; g < 2; ++g) {
+        // g = 0: every SM gets a vocabulary slice; g = 1: two row blocks per launch, so half as
+        // many slices (an even number of them: CTA pairs take two neighbouring slices)
+        SliceGeometry& geo = fs->geo[g];
+        int ctas = g == 0 ? sms : (sms / 2) & ~1;
+        if (ctas < 1) ctas = 1;
+        int per = (head.V + ctas - 1) / ctas;
+        if (per < 64) per = 64;
+        geo.tiles_per_cta = (per + kTileM - 1) / kTileM;
+        geo.tile_rows = (per + geo.tiles_per_cta - 1) / geo.tiles_per_cta;
+        geo.slice_rows = geo.tiles_per_cta * geo.tile_rows;
+        geo.n_ctas = (head.V + geo.slice_rows - 1) / geo.slice_rows;
+        const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)geo.tile_rows};
+        r = encode(&geo.tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(head.W), gdim, gstride, box,
+                   estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { delete fs; return DM_ECUDA; }
+    }
     if (cudaFuncSetAttribute(fused_head_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
             cudaSuccess ||
         cudaFuncSetAttribute(fused_head_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
@@ -723,8 +745,11 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
     fs->staging_rows = 0;
     const int widest = max_rows < kMaxNPad ? max_rows : kMaxNPad;
     SmemPlan plan;
-    if (!plan_smem(widest, fs->tiles_per_cta, &plan)) { delete fs; return DM_EUNSUPPORTED; }
-    if (plan.staged) {
+    if (!plan_smem(widest, fs->geo[0].tiles_per_cta, &plan)) { delete fs; return DM_EUNSUPPORTED; }
+    SmemPlan plan_two{};   // launches over two row blocks cut the vocabulary into longer slices
+    const bool two_staged = max_rows >= 2 * kMaxNPad && plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan_two) &&
+                            plan_two.staged;
+    if (plan.staged || two_staged) {
         fs->staging_rows = (max_rows + 15) & ~15;
         const size_t n = (size_t)fs->staging_rows * head.d * sizeof(__nv_bfloat16);
         if (cudaMalloc(&fs->staging, n) != cudaSuccess) { cudaGetLastError(); delete fs; return DM_ECUDA; }
@@ -755,23 +780,39 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out) {
     if (folded_out) *folded_out = false;
-    if (fs == nullptr || !fused_supported(head, rows) || fs->n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
-    // Every launch of a call uses the same even grid (pairs need one); a CTA whose slice lies past
-    // the end of W contributes empty partials.
-    const int grid = (fs->n_ctas + 1) & ~1;
+    if (fs == nullptr || !fused_supported(head, rows) || fs->geo[0].n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
+    // Slices of one-block launches: an even count (pairs need one); a CTA whose slice lies past the
+    // end of W contributes empty partials.
+    const int slices1 = (fs->geo[0].n_ctas + 1) & ~1;
+    const int slices2 = (fs->geo[1].n_ctas + 1) & ~1;
+    // Two full blocks of 256 paths are taken together when the launch is tensor-bound anyway: the
+    // two CTAs that share a vocabulary slice stream the same W tiles side by side, so that W comes
+    // from HBM once per 512 paths (the second reader hits L2) and a CTA runs twice as many tiles.
+    SmemPlan plan2;
+    const bool use_two = rows >= 2 * kMaxNPad && dbg_logits == nullptr &&
+                         plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan2) && plan2.pair;   // small heads: no
+    if (use_two && slices2 < slices1) {
+        // the two kinds of launch fill different numbers of slice rows of the partials: clear them
+        if (cudaMemsetAsync(partials, 0, (size_t)slices1 * rows * sizeof(unsigned long long), stream) != cudaSuccess)
+            return DM_ECUDA;
+    }
     int launches = 0;
     bool operand_staged = false;
-    for (int row0 = 0; row0 < rows; row0 += kMaxNPad) {
+    for (int row0 = 0; row0 < rows;) {
+        const int row_blocks = (use_two && rows - row0 >= 2 * kMaxNPad) ? 2 : 1;
+        const SliceGeometry& geo = fs->geo[row_blocks - 1];
+        const int grid = (row_blocks == 2 ? slices2 : slices1) * row_blocks;
         FusedParams P{};
         P.H = static_cast<const __nv_bfloat16*>(H);
         P.d = head.d; P.V = head.V;
         P.rows = rows - row0 < kMaxNPad ? rows - row0 : kMaxNPad;
         P.row0 = row0; P.rows_total = rows;
+        P.row_blocks = row_blocks;
         SmemPlan plan;
-        if (!plan_smem(P.rows, fs->tiles_per_cta, &plan)) return DM_EUNSUPPORTED;
+        if (!plan_smem(P.rows, geo.tiles_per_cta, &plan)) return DM_EUNSUPPORTED;
         P.n_pad = plan.n_pad;
         P.kb_count = head.d / kBlockK;
-        P.tiles_per_cta = fs->tiles_per_cta; P.tile_rows = fs->tile_rows; P.slice_rows = fs->slice_rows;
+        P.tiles_per_cta = geo.tiles_per_cta; P.tile_rows = geo.tile_rows; P.slice_rows = geo.slice_rows;
         P.group_tiles = plan.group_tiles; P.n_slots = plan.n_slots;
         P.nsw = plan.nsw; P.nsb = plan.nsb; P.staged = plan.staged;
         if (plan.staged && !operand_staged) {
@@ -806,19 +847,20 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
             attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
             cfg.attrs = &attr;
             cfg.numAttrs = 1;
-            if (cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, fs->tmap_w, fs->tmap_b[P.n_pad / 32 - 1], P) !=
+            if (cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, geo.tmap_w, fs->tmap_b[P.n_pad / 32 - 1], P) !=
                 cudaSuccess) {
                 cudaGetLastError();
                 return DM_ECUDA;
             }
         } else {
             fused_head_kernel<false><<<grid, kThreads, plan.total, stream>>>(
-                fs->tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : fs->tmap_w, P);
+                geo.tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : geo.tmap_w, P);
         }
         if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
         ++launches;
+        row0 += row_blocks * kMaxNPad;
     }
-    *n_slices_out = grid;
+    *n_slices_out = slices1;
     *launches_out = launches;
     return DM_OK;
 }

@@ -81,6 +81,9 @@ SMALL = [
     wl.Config("bf16_groups4", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1),
     wl.Config("bf16_groups2", d=256, V=61111, dtype=wl.BF16, B=2, T=4, K=16, p=0.2),
     wl.Config("bf16_groups_nocache", d=192, V=50000, dtype=wl.BF16, B=1, T=9, K=16, p=0.1),
+    # 600 paths: one launch that takes two blocks of 256 side by side, then one of 88
+    wl.Config("bf16_two_blocks", d=64, V=40000, dtype=wl.BF16, B=3, T=8, K=25, p=0.1),
+    wl.Config("bf16_two_blocks_exact", d=128, V=30000, dtype=wl.BF16, B=2, T=8, K=32, p=0.2),   # exactly 512
 ]
 
 
