@@ -60,7 +60,7 @@ constexpr int kPairMinNPad = DM_PAIR_MIN_NPAD;   // staged launches at least thi
 struct FusedParams {
     const __nv_bfloat16* H;
     int d, V;
-    int rows;         // paths handled by this launch (<= 256)
+    int rows;         // paths per row block of this launch (<= 256; the last block may hold fewer)
     int row0;         // first path of this launch within the call
     int rows_total;   // paths of the whole call (stride of the partials array)
     int n_pad;        // rows rounded up to a multiple of 16
@@ -132,7 +132,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int unit = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // CTA, or CTA pair
     const int rb = unit % P.row_blocks;
     const int slice = kPair ? (unit / P.row_blocks) * 2 + (int)(blockIdx.x & 1) : unit / P.row_blocks;
-    const int row0 = P.row0 + rb * kMaxNPad;     // first path of this CTA's row block within the call
+    const int row0 = P.row0 + rb * P.rows;       // first path of this CTA's row block within the call
+    const int my_rows = min(P.rows, P.rows_total - row0);   // the second block of a launch may be shorter
 
     if (threadIdx.x == 0) {
         ptx::prefetch_tensormap(&tmap_w);
@@ -157,7 +158,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             ptx::tmem_relinquish();
         }
     }
-    for (int r = threadIdx.x; r < P.rows; r += kThreads) {
+    for (int r = threadIdx.x; r < my_rows; r += kThreads) {
         RowKey k;
         bool ok = row_key(P.map, row0 + r, k);
         if (!ok) atomicExch(P.err, (uint32_t)ERR_BAD_ROW);
@@ -322,7 +323,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             ptx::bar_sync(2, kExpWarps * 32);
         }
         unsigned char* my_stage = smem + P.off_b + grp * b_stage_bytes;
-        const int n_items = P.rows * 8;            // (row, 16-byte chunk) pairs per block
+        const int n_items = my_rows * 8;           // (row, 16-byte chunk) pairs per block
         const int stride = wps * 32;               // threads working on this stage
         const int total_b = n_groups * P.kb_count;
         for (int m = grp; m < total_b; m += P.nsb) {
@@ -442,7 +443,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                     if (P.dbg_logits != nullptr && valid) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
-                            if (n0 + j < P.rows)
+                            if (n0 + j < my_rows)
                                 P.dbg_logits[(size_t)(row0 + n0 + j) * P.V + v] =
                                     s_row[n0 + j].q >= 0 ? __uint_as_float(acc[j]) * P.scale
                                                          : __uint_as_float(0x7FC00000u);
@@ -511,7 +512,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         ptx::tc_fence_before();
         ptx::bar_sync(3, 4 * n_sets * 32);
         if (warp >= kFirstExpWarp) return;      // the helpers are done; warps 2-5 finish the CTA
-        for (int n = threadIdx.x - kFirstEpiWarp * 32; n < P.rows; n += 4 * 32) {
+        for (int n = threadIdx.x - kFirstEpiWarp * 32; n < my_rows; n += 4 * 32) {
             unsigned long long b = s_best[n];
 #pragma unroll
             for (int w = 1; w < 4; ++w) {
@@ -747,7 +748,7 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
     SmemPlan plan;
     if (!plan_smem(widest, fs->geo[0].tiles_per_cta, &plan)) { delete fs; return DM_EUNSUPPORTED; }
     SmemPlan plan_two{};   // launches over two row blocks cut the vocabulary into longer slices
-    const bool two_staged = max_rows >= 2 * kMaxNPad && plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan_two) &&
+    const bool two_staged = max_rows > kMaxNPad && plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan_two) &&
                             plan_two.staged;
     if (plan.staged || two_staged) {
         fs->staging_rows = (max_rows + 15) & ~15;
@@ -788,9 +789,13 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
     // Two full blocks of 256 paths are taken together when the launch is tensor-bound anyway: the
     // two CTAs that share a vocabulary slice stream the same W tiles side by side, so that W comes
     // from HBM once per 512 paths (the second reader hits L2) and a CTA runs twice as many tiles.
+    // More than 256 paths left: two row blocks (of 256, or of half the rest) are taken in one
+    // launch.  The two CTAs that share a vocabulary slice stream the same W tiles side by side, so
+    // W comes from HBM once for both blocks (the second reader hits L2) and a CTA runs twice as
+    // many tiles.  Needs the staged operand (the longer slices never fit TMEM as one group).
     SmemPlan plan2;
-    const bool use_two = rows >= 2 * kMaxNPad && dbg_logits == nullptr &&
-                         plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan2) && plan2.pair;   // small heads: no
+    const bool use_two = rows > kMaxNPad && dbg_logits == nullptr && fs->staging != nullptr &&
+                         plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan2) && plan2.staged;
     if (use_two && slices2 < slices1) {
         // the two kinds of launch fill different numbers of slice rows of the partials: clear them
         if (cudaMemsetAsync(partials, 0, (size_t)slices1 * rows * sizeof(unsigned long long), stream) != cudaSuccess)
@@ -799,13 +804,23 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
     int launches = 0;
     bool operand_staged = false;
     for (int row0 = 0; row0 < rows;) {
-        const int row_blocks = (use_two && rows - row0 >= 2 * kMaxNPad) ? 2 : 1;
+        const int left = rows - row0;
+        int row_blocks = 1, block_rows = left < kMaxNPad ? left : kMaxNPad;
+        if (use_two && left > kMaxNPad) {
+            row_blocks = 2;
+            block_rows = left >= 2 * kMaxNPad ? kMaxNPad : (((left + 1) / 2 + 31) & ~31);   // two halves
+            SmemPlan probe;   // blocks this narrow may fit TMEM as one group: then no sharing of W
+            if (!plan_smem(block_rows, fs->geo[1].tiles_per_cta, &probe) || !probe.staged) {
+                row_blocks = 1;
+                block_rows = kMaxNPad;
+            }
+        }
         const SliceGeometry& geo = fs->geo[row_blocks - 1];
         const int grid = (row_blocks == 2 ? slices2 : slices1) * row_blocks;
         FusedParams P{};
         P.H = static_cast<const __nv_bfloat16*>(H);
         P.d = head.d; P.V = head.V;
-        P.rows = rows - row0 < kMaxNPad ? rows - row0 : kMaxNPad;
+        P.rows = block_rows;
         P.row0 = row0; P.rows_total = rows;
         P.row_blocks = row_blocks;
         SmemPlan plan;
@@ -858,7 +873,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         }
         if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
         ++launches;
-        row0 += row_blocks * kMaxNPad;
+        row0 += row_blocks * block_rows;
     }
     *n_slices_out = slices1;
     *launches_out = launches;
