@@ -21,8 +21,8 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Device-pointer entry points only enqueue work: they never
  *     synchronise, never allocate and never free.
- *   - The library allocates device memory only in dm_create / dm_set_head (its
- *     workspace) and frees it in dm_set_head / dm_destroy.
+ *   - The library allocates device memory only in dm_create, dm_set_head and
+ *     dm_enable_js (its workspace) and frees it in dm_set_head / dm_destroy.
  *   - Every function returns DM_OK or a negative status; nothing throws, aborts
  *     or prints.  A CUDA error raised by earlier asynchronous work is reported by
  *     the next call as DM_ECUDA.  A kernel that gives up on an internal wait sets
@@ -31,6 +31,7 @@
  *     (j mod 4) of Philox4x32-10(counter = (j/4, i, t, s mod 2^32),
  *     key = (seed low 32 bits, seed high 32 bits)) is < floor(p * 2^32).
  *     Results depend on (seed, s, t, i, j) only, never on batching or launch shape.
+ *     (dm_set_mask_mode can take t out of the key.)
  *   - Row order: path i of hidden row q (q = b*T + t) is "row" q*K + i.
  *   - A context is not thread-safe; use one per host thread or lock around it.
  */

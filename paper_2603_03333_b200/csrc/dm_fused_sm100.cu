@@ -1,6 +1,8 @@
-// Fused sm_100a kernel for bf16 heads: Eq. 1 masks (Philox in registers), Eq. 2 masking,
-// Eq. 3 on tcgen05 tensor cores with fp32 accumulators in TMEM, and the argmax of Sec. 3.2 in
-// the epilogue, so that neither the masked hidden rows nor any logit ever reach HBM.
+// Fused sm_100a kernel for bf16 heads: Eq. 1 masks (Philox), Eq. 2 masking, Eq. 3 on tcgen05
+// tensor cores with fp32 accumulators in TMEM, and the argmax of Sec. 3.2 in the epilogue.  W is
+// streamed from HBM once per launch and no logit is written (except on request: the debug call
+// and the JS criterion ask for them).  For calls of up to 64 paths or so the masked hidden rows
+// exist in shared memory only; for wider calls they are staged once through global memory.
 //
 // Work split.  The vocabulary is cut into one contiguous slice per CTA (one CTA per SM) and
 // each slice into equal tiles of `tile_rows` <= 128 vocabulary rows.  The MMA is "swapped": a

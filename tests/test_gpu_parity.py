@@ -309,3 +309,29 @@ def test_next_token_call(ctx, cfg, bonus):
         if not (got["tokens"] != ref["tokens"]).any() and not (got["plain"] != ref["plain"]).any():
             for key in ("counts", "hits", "accept_len", "next"):
                 assert np.array_equal(got[key], ref[key]), key
+
+
+def test_side_stream_and_head_swaps(ctx):
+    """Calls issued on a non-default stream, and a context that is pointed at one head after another
+    (fp32 -> bf16 tensor-core -> bf16 staged -> back), give what a fresh context gives."""
+    cfgs = [wl.CONFIGS["toy"],
+            wl.Config("swap_a", d=256, V=3000, dtype=wl.BF16, B=2, T=3, K=8, p=0.1),
+            wl.Config("swap_b", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1),
+            wl.Config("swap_a", d=256, V=3000, dtype=wl.BF16, B=2, T=3, K=8, p=0.1)]
+    side = torch.cuda.Stream(device=DEV)
+    for cfg in cfgs:
+        work = wl.make_workload(cfg, device=DEV)
+        torch.cuda.synchronize()
+        ctx.set_head(work.W, max_rows=cfg.rows)
+        with torch.cuda.stream(side):
+            got = ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=1)
+            again = ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=1)
+        side.synchronize()
+        assert ctx.device_error() == 0
+        fresh = pk.Context(0)
+        fresh.set_head(work.W, max_rows=cfg.rows)
+        want = to_np(fresh.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=1))
+        fresh.close()
+        for key in ("tokens", "counts", "hits", "accept_len"):
+            assert np.array_equal(got[key].cpu().numpy(), want[key]), (cfg.name, key)
+            assert np.array_equal(again[key].cpu().numpy(), want[key]), (cfg.name, key)
