@@ -121,6 +121,120 @@ js_sum_kernel(const float* __restrict__ logits, const float* __restrict__ draft_
     }
 }
 
+// ---- the same two sweeps for K <= KMAX paths with every series kept in registers --------------
+// A thread takes vocabulary entries v0 + tid, v0 + tid + 256, ...: it loads the K logits of an
+// entry once (coalesced across the block), forms the centroid and updates all K+1 running
+// results; the block is reduced once at the end.  Slot KMAX holds the centroid (first sweep) or
+// the draft distribution (second sweep).
+
+__device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
+    const float M = fmaxf(m, m2);
+    if (M == -INFINITY) { m = M; s = 0.0f; return; }
+    s = s * expf(m - M) + s2 * expf(m2 - M);
+    m = M;
+}
+
+template <int KMAX>
+__global__ void __launch_bounds__(kJsThreads)
+js_lse_reg_kernel(const float* __restrict__ logits, int V, int K, int chunk_len, int n_chunks,
+                  float2* __restrict__ part) {
+    __shared__ float2 red[kJsThreads / 32][KMAX + 1];
+    const int pos = blockIdx.y, chunk = blockIdx.x;
+    const int v0 = chunk * chunk_len, v1 = min(V, v0 + chunk_len);
+    const float* pl = logits + (size_t)pos * K * V;
+    float m[KMAX + 1], s[KMAX + 1];
+#pragma unroll
+    for (int i = 0; i <= KMAX; ++i) { m[i] = -INFINITY; s[i] = 0.0f; }
+    const float inv_k = 1.0f / (float)K;
+    for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) {
+        float c = 0.0f;
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i)
+            if (i < K) {
+                const float x = pl[(size_t)i * V + v];
+                c += x;
+                lse_merge(m[i], s[i], x, 1.0f);
+            }
+        lse_merge(m[KMAX], s[KMAX], c * inv_k, 1.0f);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int i = 0; i <= KMAX; ++i) {
+        if (i < K || i == KMAX) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1)
+                lse_merge(m[i], s[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], off), __shfl_xor_sync(0xFFFFFFFFu, s[i], off));
+            if (lane == 0) red[warp][i] = make_float2(m[i], s[i]);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i <= KMAX; i += kJsThreads) {
+        if (i < K || i == KMAX) {
+            float mm = red[0][i].x, ss = red[0][i].y;
+            for (int w = 1; w < kJsThreads / 32; ++w) lse_merge(mm, ss, red[w][i].x, red[w][i].y);
+            const int series = i == KMAX ? K : i;
+            part[((size_t)pos * (K + 1) + series) * n_chunks + chunk] = make_float2(mm, ss);
+        }
+    }
+}
+
+template <int KMAX>
+__global__ void __launch_bounds__(kJsThreads)
+js_sum_reg_kernel(const float* __restrict__ logits, const float* __restrict__ draft_prob, int V, int K,
+                  int chunk_len, int n_chunks, const float2* __restrict__ part, float* __restrict__ share) {
+    __shared__ float lse[KMAX + 1];
+    __shared__ float red[kJsThreads / 32][KMAX + 1];
+    const int pos = blockIdx.y, chunk = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int series = warp; series <= K; series += kJsThreads / 32) {   // merge the chunks' partial log-sum-exps
+        const float2* ps = part + ((size_t)pos * (K + 1) + series) * n_chunks;
+        float mm = -INFINITY, ss = 0.0f;
+        for (int c = lane; c < n_chunks; c += 32) lse_merge(mm, ss, ps[c].x, ps[c].y);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1)
+            lse_merge(mm, ss, __shfl_xor_sync(0xFFFFFFFFu, mm, off), __shfl_xor_sync(0xFFFFFFFFu, ss, off));
+        if (lane == 0) lse[series == K ? KMAX : series] = mm + logf(ss);
+    }
+    __syncthreads();
+    const int v0 = chunk * chunk_len, v1 = min(V, v0 + chunk_len);
+    const float* pl = logits + (size_t)pos * K * V;
+    const float* dp = draft_prob + (size_t)pos * V;
+    float acc[KMAX + 1];
+#pragma unroll
+    for (int i = 0; i <= KMAX; ++i) acc[i] = 0.0f;
+    const float inv_k = 1.0f / (float)K, lse_c = lse[KMAX];
+    for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) {
+        float x[KMAX];
+        float c = 0.0f;
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i)
+            if (i < K) { x[i] = pl[(size_t)i * V + v]; c += x[i]; }
+        const float lq = c * inv_k - lse_c;                       // log pbar[v]
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i)
+            if (i < K) acc[i] += js_term(x[i] - lse[i], lq);
+        const float P = dp[v];
+        acc[KMAX] += js_term(P > 0.0f ? logf(P) : -INFINITY, lq);
+    }
+#pragma unroll
+    for (int i = 0; i <= KMAX; ++i) {
+        if (i < K || i == KMAX) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc[i] += __shfl_xor_sync(0xFFFFFFFFu, acc[i], off);
+            if (lane == 0) red[warp][i] = acc[i];
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i <= KMAX; i += kJsThreads) {
+        if (i < K || i == KMAX) {
+            float t = 0.0f;
+            for (int w = 0; w < kJsThreads / 32; ++w) t += red[w][i];
+            const int series = i == KMAX ? K : i;
+            share[((size_t)pos * (K + 1) + series) * n_chunks + chunk] = 0.5f * t;
+        }
+    }
+}
+
 // Algorithm 1 and the left-to-right scan for one sequence; also exports the divergences.
 __global__ void __launch_bounds__(kJsThreads)
 js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, const int32_t* __restrict__ tokens,
@@ -128,12 +242,14 @@ js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, co
                  int32_t* __restrict__ out_accept_len) {
     extern __shared__ int32_t ok[];   // [T]
     const int b = blockIdx.x;
-    // divergences: one thread per (position, series), chunks summed in double
-    for (int x = threadIdx.x; x < T * (K + 1); x += kJsThreads) {
+    // divergences: one warp per (position, series), lanes over the chunks, summed in double
+    for (int x = threadIdx.x >> 5; x < T * (K + 1); x += kJsThreads / 32) {
         const size_t idx = (size_t)b * T * (K + 1) + x;
         double acc = 0.0;
-        for (int c = 0; c < n_chunks; ++c) acc += (double)share[idx * n_chunks + c];
-        out_js[idx] = (float)acc;
+        for (int c = threadIdx.x & 31; c < n_chunks; c += 32) acc += (double)share[idx * n_chunks + c];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+        if ((threadIdx.x & 31) == 0) out_js[idx] = (float)acc;
     }
     __syncthreads();
     for (int t = threadIdx.x; t < T; t += kJsThreads) {
@@ -175,9 +291,20 @@ int launch_js(const float* logits, const float* draft_prob, float* workspace, in
     float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
     if ((size_t)(K + 1 + chunk_len) * sizeof(float) > 40 * 1024 || (size_t)T * sizeof(int32_t) > 40 * 1024) return DM_EUNSUPPORTED;
     dim3 grid((unsigned)n_chunks, (unsigned)n_pos);
-    js_lse_kernel<<<grid, kJsThreads, chunk_len * sizeof(float), stream>>>(logits, V, K, chunk_len, n_chunks, part);
-    js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K, chunk_len,
-                                                                      n_chunks, part, share);
+    if (K <= 8) {
+        js_lse_reg_kernel<8><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
+        js_sum_reg_kernel<8><<<grid, kJsThreads, 0, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share);
+    } else if (K <= 16) {
+        js_lse_reg_kernel<16><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
+        js_sum_reg_kernel<16><<<grid, kJsThreads, 0, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share);
+    } else if (K <= 32) {
+        js_lse_reg_kernel<32><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
+        js_sum_reg_kernel<32><<<grid, kJsThreads, 0, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share);
+    } else {   // more paths than fit in registers: one series at a time
+        js_lse_kernel<<<grid, kJsThreads, chunk_len * sizeof(float), stream>>>(logits, V, K, chunk_len, n_chunks, part);
+        js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K,
+                                                                                      chunk_len, n_chunks, part, share);
+    }
     js_accept_kernel<<<B, kJsThreads, T * sizeof(int32_t), stream>>>(share, n_chunks, T, K, tokens, draft, out_js,
                                                                   out_js_ok, out_accept_len);
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
