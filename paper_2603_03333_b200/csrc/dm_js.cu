@@ -77,9 +77,11 @@ __device__ __forceinline__ float js_term(float lp, float lq) {
     const float hi = fmaxf(lp, lq), lo = fminf(lp, lq);
     if (hi == -INFINITY) return 0.0f;
     const float a = lo - hi;                                  // may be -inf
-    const float r = -logf(0.5f + 0.5f * expf(a));             // log(P_hi / M), in [0, log 2]
-    float t = expf(hi) * r;
-    if (a > -INFINITY) t += expf(lo) * (a + r);               // log(P_lo / M) = a + r
+    // fast intrinsics: the logarithm's argument lies in [0.5, 1], where __logf is good to ~4e-7
+    // absolute, and every exponent is <= 0; the errors are weighted by probabilities that sum to 1
+    const float r = -__logf(0.5f + 0.5f * __expf(a));         // log(P_hi / M), in [0, log 2]
+    float t = __expf(hi) * r;
+    if (a > -INFINITY) t += __expf(lo) * (a + r);             // log(P_lo / M) = a + r
     return t;
 }
 
@@ -130,7 +132,9 @@ js_sum_kernel(const float* __restrict__ logits, const float* __restrict__ draft_
 __device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
     const float M = fmaxf(m, m2);
     if (M == -INFINITY) { m = M; s = 0.0f; return; }
-    s = s * expf(m - M) + s2 * expf(m2 - M);
+    // fast exponentials: relative error ~1e-7 per term of a sum of positive terms, far inside the
+    // tolerance of the divergences (the arguments are <= 0)
+    s = s * __expf(m - M) + s2 * __expf(m2 - M);
     m = M;
 }
 
@@ -161,10 +165,13 @@ js_lse_reg_kernel(const float* __restrict__ logits, int V, int K, int chunk_len,
 #pragma unroll
     for (int i = 0; i <= KMAX; ++i) {
         if (i < K || i == KMAX) {
+            float M = m[i];
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1)
-                lse_merge(m[i], s[i], __shfl_xor_sync(0xFFFFFFFFu, m[i], off), __shfl_xor_sync(0xFFFFFFFFu, s[i], off));
-            if (lane == 0) red[warp][i] = make_float2(m[i], s[i]);
+            for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
+            float t = M == -INFINITY ? 0.0f : s[i] * __expf(m[i] - M);   // one rescale, then a plain sum
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
+            if (lane == 0) red[warp][i] = make_float2(M, t);
         }
     }
     __syncthreads();
