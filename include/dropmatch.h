@@ -160,6 +160,27 @@ int dropmatch_verify_js(dm_ctx* ctx, const void* H, const int32_t* draft, const 
                         int32_t* out_counts, float* out_js, int32_t* out_js_ok, int32_t* out_accept_len,
                         void* stream);
 
+/* Vocabulary-sharded heads (the deployment of Sec. 4.1 is tensor-parallel: every GPU holds a
+ * slice of the LM head).  A context whose head is rows [offset, offset+V) of the full head reports
+ * global token ids after dm_set_vocab_offset(ctx, offset) (call it after dm_set_head; default 0).
+ * The masks are keyed on indices only, so every shard draws the same masks without any exchange.
+ *
+ * dropmatch_partial_best runs Eq. 1-3 and the vocabulary reduction on this context's head and
+ * writes one packed word per path, out_packed[B*T*K] (device): (ordered fp32 key of the best logit
+ * << 32) | (2^32-1 - token id).  The elementwise maximum of such arrays from all shards is the
+ * result for the full head (equal logits resolve to the smaller token id).
+ *
+ * dropmatch_finalize_packed takes n_parts such arrays back to back, packed[n_parts][B*T*K]
+ * (device) -- the layout an all-gather over the shards produces -- merges them and runs the
+ * histogram and the acceptance scan as dropmatch_verify_batched does.  Needs no head.
+ * Both only enqueue work on `stream`. */
+int dm_set_vocab_offset(dm_ctx* ctx, int offset);
+int dropmatch_partial_best(dm_ctx* ctx, const void* H, int B, int T, int K, float p, uint64_t seed,
+                           uint64_t seq_base, uint64_t* out_packed, void* stream);
+int dropmatch_finalize_packed(dm_ctx* ctx, const uint64_t* packed, int n_parts, const int32_t* draft, int B, int T,
+                              int K, int rule, int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
+                              int32_t* out_accept_len, void* stream);
+
 /* The paper has no counterpart to this entry point; it exists for the way the library gets
  * deployed.  Some hosts of this code cannot ask CUDA for device memory at the time they verify:
  * a serving process that hands all of HBM to its own pool at start-up (a later cudaMalloc fails

@@ -4,4 +4,5 @@ The work is done by libdropmatch.so (CUDA, C ABI in include/dropmatch.h); `bindi
 torch tensors into it and `workloads` draws seeded synthetic inputs.
 """
 from . import binding, workloads  # noqa: F401
+from . import vocab_parallel  # noqa: F401
 from .binding import Context, DropMatchError  # noqa: F401

@@ -30,6 +30,9 @@ SIGNATURES = {
     "dm_set_head": (_ci, [_vp, _vp, _ci, _ci, _ci, _ci, _ci]),
     "dm_set_impl": (_ci, [_vp, _ci]),
     "dm_set_mask_mode": (_ci, [_vp, _ci]),
+    "dm_set_vocab_offset": (_ci, [_vp, _ci]),
+    "dropmatch_partial_best": (_ci, [_vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
+    "dropmatch_finalize_packed": (_ci, [_vp, _vp, _ci, _vp, _ci, _ci, _ci, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _u64, _ci, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_next": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
@@ -155,6 +158,35 @@ class Context:
 
     def set_mask_mode(self, mode: int):
         _check(lib().dm_set_mask_mode(self._h, mode), "dm_set_mask_mode")
+
+    # -- vocabulary-sharded heads
+    def set_vocab_offset(self, offset: int):
+        _check(lib().dm_set_vocab_offset(self._h, offset), "dm_set_vocab_offset")
+
+    def partial_best(self, H, K, p, seed, seq_base=0):
+        """-> int64 tensor [B*T*K] holding the packed (key, inverted token id) words bit for bit."""
+        B, T, _ = H.shape
+        _dev(H, self._tdtype(), "H")
+        out = torch.empty((B * T * K,), dtype=torch.int64, device=self.device)
+        _check(lib().dropmatch_partial_best(self._h, _ptr(H), B, T, K, p, seed, seq_base, _ptr(out),
+                                            _stream(self.device)), "dropmatch_partial_best")
+        return out
+
+    def finalize_packed(self, packed, draft, K, rule=RULE_NAIVE):
+        """packed: int64 [n_parts, B*T*K] (or [B*T*K]); draft[B,T] -> the outputs of verify_batched."""
+        _dev(draft, torch.int32, "draft")
+        B, T = draft.shape
+        if packed.dim() == 1:
+            packed = packed.unsqueeze(0)
+        _dev(packed, torch.int64, "packed")
+        if packed.shape[1] != B * T * K:
+            raise TypeError("packed must have B*T*K words per part")
+        out = self.alloc_outputs(B, T, K)
+        _check(lib().dropmatch_finalize_packed(self._h, _ptr(packed), packed.shape[0], _ptr(draft), B, T, K, rule,
+                                               _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["hits"]),
+                                               _ptr(out["accept_len"]), _stream(self.device)),
+               "dropmatch_finalize_packed")
+        return out
 
     # -- dropmatch_verify
     def verify(self, H, draft, K, p, seed, rule=RULE_NAIVE):

@@ -10,7 +10,7 @@ using namespace dm;
 
 struct dm_ctx {
     int device = 0;
-    HeadDesc head{nullptr, 0, 0, 0};
+    HeadDesc head{nullptr, 0, 0, 0, 0};
     bool has_head = false;
     int max_rows = 0, max_hidden = 0;
     int impl = DM_IMPL_AUTO;
@@ -220,7 +220,7 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
     }
     c->pin_out_dev = static_cast<int32_t*>(out_dev);
     c->ws_bytes = n_part + n_in;
-    c->head = HeadDesc{W, V, d, dtype};
+    c->head = HeadDesc{W, V, d, dtype, 0};
     c->max_rows = max_rows;
     c->max_hidden = max_hidden_rows;
     size_t fused_bytes = 0;
@@ -235,6 +235,65 @@ int dm_set_impl(dm_ctx* c, int impl) {
     if (c == nullptr || impl < DM_IMPL_AUTO || impl > DM_IMPL_TCGEN05) return DM_EINVAL;
     c->impl = impl;
     return DM_OK;
+}
+
+int dm_set_vocab_offset(dm_ctx* c, int offset) {
+    if (c == nullptr) return DM_EINVAL;
+    if (!c->has_head) return DM_ENOHEAD;
+    if (offset < 0 || (long long)offset + c->head.V > 0x7FFFFFFFll) return DM_EINVAL;
+    c->head.v_offset = offset;
+    return DM_OK;
+}
+
+int dropmatch_partial_best(dm_ctx* c, const void* H, int B, int T, int K, float p, uint64_t seed,
+                           uint64_t seq_base, uint64_t* out_packed, void* stream) {
+    int st = check_common(c, H, B, T, K);
+    if (st != DM_OK) return st;
+    if (out_packed == nullptr) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    const int rows = B * T * K;
+    if (rows > c->max_rows) return DM_EWORKSPACE;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};
+    int impl;
+    st = pick_impl(c, rows, &impl);
+    if (st != DM_OK) return st;
+    int n_slices = 0, launches = 1;
+    if (impl == DM_IMPL_TCGEN05)   // no finalize arguments: the kernels leave per-slice partials
+        st = fused_launch(c->fused, c->head, H, B * T, rows, map, mk, &n_slices, c->partials, nullptr, c->err, s,
+                          &launches);
+    else
+        st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, s);
+    if (st != DM_OK) return st;
+    st = launch_merge_partials(c->partials, n_slices, rows, reinterpret_cast<unsigned long long*>(out_packed), s);
+    if (st != DM_OK) return st;
+    c->last_impl = impl;
+    c->last_launches = launches + 1;
+    return DM_OK;
+}
+
+int dropmatch_finalize_packed(dm_ctx* c, const uint64_t* packed, int n_parts, const int32_t* draft, int B, int T,
+                              int K, int rule, int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
+                              int32_t* out_accept_len, void* stream) {
+    if (c == nullptr || packed == nullptr || draft == nullptr || out_tokens == nullptr || out_counts == nullptr ||
+        out_accept_len == nullptr)
+        return DM_EINVAL;
+    if (n_parts < 1 || n_parts > 4096 || B < 1 || T < 1 || K < 1 || K > kMaxK) return DM_EINVAL;
+    if ((long long)B * T * K > 0x3FFFFFFFll) return DM_EINVAL;
+    if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = T; fa.K = K; fa.rule = rule;
+    fa.draft = draft; fa.out_hits = out_draft_hits;
+    fa.N = 0;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    return launch_finalize(reinterpret_cast<const unsigned long long*>(packed), n_parts, B * T * K, fa,
+                           static_cast<cudaStream_t>(stream));
 }
 
 int dm_set_mask_mode(dm_ctx* c, int mode) {

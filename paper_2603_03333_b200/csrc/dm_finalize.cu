@@ -11,6 +11,39 @@ finalize_kernel(const unsigned long long* __restrict__ partials, int n_slices, i
     finalize_sequence(partials, n_slices, rows, a, (int)blockIdx.x, sm, (int)threadIdx.x, (int)blockDim.x, BlockSync{});
 }
 
+// One packed word per row: the maximum over the slices (argmax with the smallest index on ties).
+__global__ void __launch_bounds__(256)
+merge_partials_kernel(const unsigned long long* __restrict__ partials, int n_slices, int rows,
+                      unsigned long long* __restrict__ out_packed) {
+    const int warp = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    const int x0 = warp * 4;   // four rows per warp: their loads overlap
+    if (x0 >= rows) return;
+    unsigned long long best[4] = {0ull, 0ull, 0ull, 0ull};
+    for (int s = lane; s < n_slices; s += 32)
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (x0 + u < rows) {
+                unsigned long long c = __ldcg(partials + (size_t)s * rows + x0 + u);
+                best[u] = c > best[u] ? c : best[u];
+            }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best[u], off);
+            best[u] = o > best[u] ? o : best[u];
+        }
+        if (lane == 0 && x0 + u < rows) out_packed[x0 + u] = best[u];
+    }
+}
+
+int launch_merge_partials(const unsigned long long* partials, int n_slices, int rows,
+                          unsigned long long* out_packed, cudaStream_t stream) {
+    const int warps = (rows + 3) / 4;
+    merge_partials_kernel<<<(warps * 32 + 255) / 256, 256, 0, stream>>>(partials, n_slices, rows, out_packed);
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+}
+
 size_t finalize_smem_bytes(int T, int K, int N) {
     size_t extra = N > 0 ? 2 * (size_t)N : (size_t)T;
     return ((size_t)T * K + extra) * sizeof(int32_t);

@@ -62,6 +62,7 @@ constexpr int kPairMinNPad = DM_PAIR_MIN_NPAD;   // staged launches at least thi
 struct FusedParams {
     const __nv_bfloat16* H;
     int d, V;
+    int v_offset;     // added to every token id (vocabulary-sharded heads)
     int rows;         // paths per row block of this launch (<= 256; the last block may hold fewer)
     int row0;         // first path of this launch within the call
     int rows_total;   // paths of the whole call (stride of the partials array)
@@ -454,7 +455,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                 unsigned long long p16[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    p16[j] = best[j] != neg_inf ? pack_best(float_key(best[j]), (uint32_t)bv[j]) : 0ull;
+                    p16[j] = best[j] != neg_inf ? pack_best(float_key(best[j]), (uint32_t)(bv[j] + P.v_offset)) : 0ull;
                 unsigned long long p8[8], p4[4], p2[2], p1;
                 {
                     const bool up = (lane & 16) != 0;
@@ -821,7 +822,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         const int grid = (row_blocks == 2 ? slices2 : slices1) * row_blocks;
         FusedParams P{};
         P.H = static_cast<const __nv_bfloat16*>(H);
-        P.d = head.d; P.V = head.V;
+        P.d = head.d; P.V = head.V; P.v_offset = head.v_offset;
         P.rows = block_rows;
         P.row0 = row0; P.rows_total = rows;
         P.row_blocks = row_blocks;

@@ -17,6 +17,7 @@ constexpr int kMaxK = 1024;
 struct HeadDesc {
     const void* W;
     int V, d, dtype;
+    int v_offset;   // added to every token id: first vocabulary row of this head within a sharded one
 };
 
 // Per-call mask parameters (Eq. 1, Eq. 2).
@@ -48,6 +49,10 @@ struct FinalizeArgs {
     int32_t* out_counts;         // [B,T,K]
     int32_t* out_accept_len;     // [B]
 };
+
+// Reduce the per-slice partial argmaxes to one packed word per row (no histogram, no acceptance).
+int launch_merge_partials(const unsigned long long* partials, int n_slices, int rows,
+                          unsigned long long* out_packed, cudaStream_t stream);
 
 int launch_simt(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
                 int* n_slices_out, unsigned long long* partials, float* dbg_logits, uint32_t* err,

@@ -96,7 +96,7 @@ extern "C" int dropmatch_verify_batched_static(int device, const void* W, int V,
 
         static_scratch_reset_kernel<<<1, 1, 0, s>>>();
         if (cudaGetLastError() != cudaSuccess) { st = DM_ECUDA; break; }
-        HeadDesc head{W, V, d, dtype};
+        HeadDesc head{W, V, d, dtype, 0};
         RowMap map{nullptr, K, T, B, (uint32_t)seq_base};
         int n_slices = 0;
         st = launch_simt(head, H, (int)rows, map, mk, &n_slices, partials, nullptr, err, s);
