@@ -21,6 +21,8 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Device-pointer entry points only enqueue work: they never
  *     synchronise, never allocate and never free.
+ *     The context-based verify calls (dropmatch_verify, _batched, _tree, _batched_next, _js)
+ *     can therefore be captured into a CUDA graph; the seed and all sizes are then fixed.
  *   - The library allocates device memory only in dm_create, dm_set_head and
  *     dm_enable_js (its workspace) and frees it in dm_set_head / dm_destroy.
  *   - Every function returns DM_OK or a negative status; nothing throws, aborts

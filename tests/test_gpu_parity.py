@@ -335,3 +335,29 @@ def test_side_stream_and_head_swaps(ctx):
         for key in ("tokens", "counts", "hits", "accept_len"):
             assert np.array_equal(got[key].cpu().numpy(), want[key]), (cfg.name, key)
             assert np.array_equal(again[key].cpu().numpy(), want[key]), (cfg.name, key)
+
+
+@pytest.mark.parametrize("cfg", [
+    wl.Config("graph_a", d=256, V=3000, dtype=wl.BF16, B=2, T=3, K=8, p=0.1),            # one launch per call
+    wl.Config("graph_b", d=128, V=60000, dtype=wl.BF16, B=2, T=8, K=25, p=0.1),          # 400 paths: staged, two row blocks
+], ids=lambda c: c.name)
+def test_verify_call_in_a_cuda_graph(ctx, cfg):
+    """The device-pointer entry points only enqueue work (no allocation, no synchronisation), so a
+    call can be captured into a CUDA graph and replayed; every replay gives the eager result."""
+    work = wl.make_workload(cfg, device=DEV)
+    ctx.set_head(work.W, max_rows=cfg.rows)
+    want = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=6))
+    out = ctx.alloc_outputs(cfg.B, cfg.T, cfg.K)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=6, out=out)
+    for _ in range(3):
+        for t in out.values():
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        got = to_np(out)
+        for key in ("tokens", "counts", "hits", "accept_len"):
+            assert np.array_equal(got[key], want[key]), key
+    assert ctx.device_error() == 0
