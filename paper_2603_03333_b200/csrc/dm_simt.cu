@@ -115,13 +115,11 @@ simt_head_kernel(const T* __restrict__ W, const T* __restrict__ H, int V, int d,
     }
 }
 
-template <typename T>
-static int launch_simt_t(const HeadDesc& head, const void* H, int rows, const RowMap& map,
-                         const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
-                         float* dbg_logits, uint32_t* err, cudaStream_t stream) {
-    constexpr int RC = 8;
+template <typename T, int RC>
+static int launch_simt_rc(const HeadDesc& head, const void* H, int rows, const RowMap& map,
+                          const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
+                          float* dbg_logits, uint32_t* err, cudaStream_t stream) {
     const size_t smem = (size_t)RC * head.d * sizeof(T);
-    if (smem > 200 * 1024) return DM_EUNSUPPORTED;
     int v_per_block = (head.V + kSimtMaxSlices - 1) / kSimtMaxSlices;
     if (v_per_block < 8) v_per_block = 8;
     const int n_slices = (head.V + v_per_block - 1) / v_per_block;
@@ -134,6 +132,24 @@ static int launch_simt_t(const HeadDesc& head, const void* H, int rows, const Ro
     if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
     *n_slices_out = n_slices;
     return DM_OK;
+}
+
+// Eight masked rows at a time fit shared memory up to d = 12800 (bf16) or 6400 (fp32); longer
+// hidden sizes take four, two or one row at a time (W is then re-read from L2 more often).
+template <typename T>
+static int launch_simt_t(const HeadDesc& head, const void* H, int rows, const RowMap& map,
+                         const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
+                         float* dbg_logits, uint32_t* err, cudaStream_t stream) {
+    const size_t row_bytes = (size_t)head.d * sizeof(T), limit = 200 * 1024;
+    if (8 * row_bytes <= limit)
+        return launch_simt_rc<T, 8>(head, H, rows, map, mk, n_slices_out, partials, dbg_logits, err, stream);
+    if (4 * row_bytes <= limit)
+        return launch_simt_rc<T, 4>(head, H, rows, map, mk, n_slices_out, partials, dbg_logits, err, stream);
+    if (2 * row_bytes <= limit)
+        return launch_simt_rc<T, 2>(head, H, rows, map, mk, n_slices_out, partials, dbg_logits, err, stream);
+    if (row_bytes <= limit)
+        return launch_simt_rc<T, 1>(head, H, rows, map, mk, n_slices_out, partials, dbg_logits, err, stream);
+    return DM_EUNSUPPORTED;
 }
 
 int launch_simt(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,

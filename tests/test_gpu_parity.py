@@ -250,6 +250,10 @@ EDGE = [
     # widest single launch exactly (256 paths) and one more (257)
     wl.Config("edge_rows256", d=64, V=40000, dtype=wl.BF16, B=1, T=8, K=32, p=0.1),
     wl.Config("edge_rows257", d=64, V=1000, dtype=wl.BF16, B=1, T=1, K=257, p=0.1),
+    # a vocabulary so large that a slice has 16 tiles even at 24 paths (staged operand, many groups)
+    wl.Config("edge_big_v", d=64, V=300000, dtype=wl.BF16, B=1, T=3, K=8, p=0.1),
+    # a long hidden size (256 blocks of 64) on a small vocabulary
+    wl.Config("edge_long_d", d=16384, V=700, dtype=wl.BF16, B=1, T=2, K=8, p=0.1),
     # fp32 head whose hidden size is the minimum the CUDA-core kernel takes
     wl.Config("edge_f32_d4", d=4, V=50, dtype=wl.F32, B=1, T=2, K=16, p=0.5, draft_mode="toy"),
 ]
