@@ -20,6 +20,7 @@
  *   Eq. 6 (majority) accept iff draft token equals the most frequent path token
  *   Sec. 2 ("Lossless Speculative Decoding" paragraph): a rejection rejects all
  *                    later positions -> accepted length = leading run of accepts.
+ *   Eq. 4, Eq. 5, Algorithm 1: centroid distribution, Jensen-Shannon test, JS-else-majority.
  *   Sec. 4.4         tree drafts: candidates under one parent share that parent's
  *                    target distribution; naive rule per node; the result is the
  *                    longest accepted root-to-leaf path.
@@ -28,7 +29,11 @@
  * independent Python-integer Philox, Bernoulli closed forms, p=0 == fp64 GEMV
  * + greedy verification, K=1 single path, brute force over all 16 masks at d=4,
  * linearity identity, scale invariance, first-reject-stops, nested-K
- * monotonicity, batched == singles, chain == path-shaped tree.
+ * monotonicity, batched == singles, chain == path-shaped tree.  JS criterion (Eq. 4, Eq. 5,
+ * Algorithm 1): scipy's Jensen-Shannon distance, relative entropy and softmax, closed forms,
+ * a scipy restatement of Algorithm 1 with both outcomes, p=0 collapse onto the centroid.
+ * Next-token call: library fp64 GEMV argmax and a brute-force scan.  Shared masks: equal hidden
+ * rows decode alike path by path, position t equals a one-position call.
  * Parity unpinned: the paper's printed aggregates (tau, agreement ratios) need
  * the authors' models and datasets and cannot pin anything here.
  */
