@@ -227,6 +227,17 @@ int dropmatch_verify_tree(dm_ctx* ctx, const void* H, const int32_t* node_token,
                           int32_t* out_tokens, int32_t* out_counts, int32_t* out_node_ok,
                           int32_t* out_best_node, int32_t* out_accept_len, void* stream);
 
+/* dropmatch_verify_tree plus, in the same pass over W, the target's own greedy token of every
+ * hidden row (one more path without dropout, as in dropmatch_verify_batched_next):
+ * out_plain_tokens[B,N_h].  The token to emit after the accepted path is the entry of the hidden
+ * row that the best node owns (the caller knows which row that is; it need not exist for a leaf).
+ * Counts B*N_h*(K+1) rows against max_rows.  K <= 1023. */
+int dropmatch_verify_tree_next(dm_ctx* ctx, const void* H, const int32_t* node_token, const int32_t* node_parent,
+                               const int32_t* node_hrow, int B, int N_h, int N, int K, float p, uint64_t seed,
+                               uint64_t seq_base, int rule, int32_t* out_tokens, int32_t* out_counts,
+                               int32_t* out_node_ok, int32_t* out_best_node, int32_t* out_accept_len,
+                               int32_t* out_plain_tokens, void* stream);
+
 /* Debug: full logits (Eq. 3 with Eq. 2's scale) of selected paths, computed by the same kernel
  * family a verify call would use.  H[B,T,d]; row_sel[n_sel,3] holds (b, t, i) triples with
  * 0 <= b < B, 0 <= t < T, i >= 0 (checked on the device: a bad triple yields a row of NaN);

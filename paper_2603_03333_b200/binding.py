@@ -44,6 +44,8 @@ SIGNATURES = {
     "dropmatch_verify_js": (_ci, [_vp, _vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_tree": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
                                     _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_tree_next": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
+                                         _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_debug_masks": (_ci, [_vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_device_error": (_ci, [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]),
@@ -289,6 +291,24 @@ class Context:
                                            B, N_h, N, K, p, seed, seq_base, rule, _ptr(out["tokens"]),
                                            _ptr(out["counts"]), _ptr(out["node_ok"]), _ptr(out["best_node"]),
                                            _ptr(out["accept_len"]), _stream(self.device)), "dropmatch_verify_tree")
+        return out
+
+    def verify_tree_next(self, H, node_token, node_parent, node_hrow, K, p, seed, seq_base=0, rule=RULE_NAIVE):
+        """verify_tree plus plain[B,N_h]: the undropped greedy token of every hidden row."""
+        B, N_h, _ = H.shape
+        N = node_token.shape[1]
+        _dev(H, self._tdtype(), "H")
+        for name, t in (("node_token", node_token), ("node_parent", node_parent), ("node_hrow", node_hrow)):
+            _dev(t, torch.int32, name)
+        i32 = dict(dtype=torch.int32, device=self.device)
+        out = dict(tokens=torch.empty((B, N_h, K), **i32), counts=torch.empty((B, N_h, K), **i32),
+                   node_ok=torch.empty((B, N), **i32), best_node=torch.empty((B,), **i32),
+                   accept_len=torch.empty((B,), **i32), plain=torch.empty((B, N_h), **i32))
+        _check(lib().dropmatch_verify_tree_next(self._h, _ptr(H), _ptr(node_token), _ptr(node_parent),
+                                                _ptr(node_hrow), B, N_h, N, K, p, seed, seq_base, rule,
+                                                _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["node_ok"]),
+                                                _ptr(out["best_node"]), _ptr(out["accept_len"]), _ptr(out["plain"]),
+                                                _stream(self.device)), "dropmatch_verify_tree_next")
         return out
 
     # -- debug

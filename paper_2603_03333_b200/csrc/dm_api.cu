@@ -488,6 +488,33 @@ int dropmatch_verify_tree(dm_ctx* c, const void* H, const int32_t* node_token, c
     return run_verify(c, H, B * N_h * K, map, mk, fa, static_cast<cudaStream_t>(stream));
 }
 
+int dropmatch_verify_tree_next(dm_ctx* c, const void* H, const int32_t* node_token, const int32_t* node_parent,
+                               const int32_t* node_hrow, int B, int N_h, int N, int K, float p, uint64_t seed,
+                               uint64_t seq_base, int rule, int32_t* out_tokens, int32_t* out_counts,
+                               int32_t* out_node_ok, int32_t* out_best_node, int32_t* out_accept_len,
+                               int32_t* out_plain_tokens, void* stream) {
+    int st = check_common(c, H, B, N_h, K);
+    if (st != DM_OK) return st;
+    if (N < 1 || N > (1 << 20) || K + 1 > kMaxK) return DM_EINVAL;
+    if (node_token == nullptr || node_parent == nullptr || node_hrow == nullptr || out_tokens == nullptr ||
+        out_counts == nullptr || out_best_node == nullptr || out_accept_len == nullptr || out_plain_tokens == nullptr)
+        return DM_EINVAL;
+    if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
+    if ((long long)B * N_h * (K + 1) > 0x3FFFFFFFll) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    RowMap map{nullptr, K, N_h, B, (uint32_t)seq_base, c->mask_mode, 1};
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = N_h; fa.K = K; fa.rule = rule;
+    fa.plain = 1; fa.out_plain = out_plain_tokens;
+    fa.N = N; fa.node_token = node_token; fa.node_parent = node_parent; fa.node_hrow = node_hrow;
+    fa.out_node_ok = out_node_ok; fa.out_best_node = out_best_node;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    return run_verify(c, H, B * N_h * (K + 1), map, mk, fa, static_cast<cudaStream_t>(stream));
+}
+
 int dm_debug_logits(dm_ctx* c, const void* H, int B, int T, const int32_t* row_sel, int n_sel, float p,
                     uint64_t seed, uint64_t seq_base, float* out_logits, void* stream) {
     if (c == nullptr || H == nullptr || row_sel == nullptr || out_logits == nullptr) return DM_EINVAL;

@@ -365,3 +365,27 @@ def test_verify_call_in_a_cuda_graph(ctx, cfg):
         for key in ("tokens", "counts", "hits", "accept_len"):
             assert np.array_equal(got[key], want[key]), key
     assert ctx.device_error() == 0
+
+
+def test_tree_with_plain_tokens(ctx):
+    """dropmatch_verify_tree_next: the tree results equal dropmatch_verify_tree's, and the extra
+    unmasked path of every hidden row is the oracle's plain greedy token (outside near-ties)."""
+    cfg = wl.Config("tree_next", d=256, V=4000, dtype=wl.BF16, B=3, T=0, K=8, p=0.15, kind="tree", N=25)
+    work = wl.make_workload(cfg, device=DEV)
+    cfg = work.cfg
+    ctx.set_head(work.W, max_rows=cfg.B * cfg.T * (cfg.K + 1))
+    Wn, Hn = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H)
+    dummy = np.zeros((cfg.B, cfg.T), dtype=np.int32)
+    plain_ref = oracle.verify_batched_next(Wn, cfg.dtype, Hn, dummy, 1, 0.0, SEED)     # only its plain tokens are used
+    for impl in _impls(ctx, cfg):
+        ctx.set_impl(impl)
+        base = to_np(ctx.verify_tree(work.H, work.node_token, work.node_parent, work.node_hrow, cfg.K, cfg.p, SEED,
+                                     seq_base=2))
+        got = to_np(ctx.verify_tree_next(work.H, work.node_token, work.node_parent, work.node_hrow, cfg.K, cfg.p,
+                                         SEED, seq_base=2))
+        ctx.set_impl(binding.IMPL_AUTO)
+        assert ctx.device_error() == 0
+        for key in ("tokens", "counts", "node_ok", "best_node", "accept_len"):
+            assert np.array_equal(got[key], base[key]), key
+        bad = (got["plain"] != plain_ref["plain"]) & (plain_ref["plain_gap"] >= NEAR_TIE)
+        assert not bad.any()
