@@ -215,6 +215,17 @@ def run_cuda(args):
     ctx.profile_head(False)
     head_ms_avg = ms_sum / max(1, n_prof)
 
+    # read-only HBM ceiling of this machine, measured live: a plain streaming read of W (larger than L2)
+    for _ in range(3):
+        ctx.debug_read_stream(work.W)
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r0.record()
+    for _ in range(20):
+        ctx.debug_read_stream(work.W)
+    r1.record()
+    torch.cuda.synchronize()
+    read_only_gbs = work.W.numel() * work.W.element_size() * 20 / (r0.elapsed_time(r1) * 1e-3) / 1e9
+
     elem = 2 if cfg.dtype == wl.BF16 else 4
     alg_bytes = (cfg.V * cfg.d + cfg.B * cfg.T * cfg.d) * elem
     alg_flops = 2.0 * cfg.rows * cfg.V * cfg.d
@@ -230,7 +241,8 @@ def run_cuda(args):
         roofline = dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
                         frac=achieved / peaks["bf16_tflops"], traffic=NCU_TRAFFIC_BYTES.get(args.workload),
                         peak_source=f"of {peaks['source']} (cuBLAS bf16, burst)", algorithmic_flops=alg_flops)
-    roofline.update(kernel="fused_head_kernel", kernel_ms=head_ms_avg,
+    roofline.update(kernel="fused_head_kernel", kernel_ms=head_ms_avg, read_only_stream_gbs=read_only_gbs,
+                    frac_of_read_only_stream=(alg_bytes / (head_ms_avg * 1e-3) / 1e9) / read_only_gbs,
                     whole_call_gbs=alg_bytes / (ms_step * 1e-3) / 1e9)
 
     # end to end through the host-buffer entry point: H2D of H and draft, D2H of all results, per step

@@ -250,6 +250,11 @@ int dm_debug_logits(dm_ctx* ctx, const void* H, int B, int T, const int32_t* row
 int dm_debug_masks(dm_ctx* ctx, int B, int T, int K, int d, float p, uint64_t seed,
                    uint64_t seq_base, uint32_t* out_bits, void* stream);
 
+/* Measurement aid: enqueues one read-only pass over `bytes` bytes at device pointer `ptr` (16-byte
+ * aligned; the bytes beyond a multiple of 16 are not read).  Timed over a buffer much larger than
+ * L2 it gives the read-only HBM rate of the part, the ceiling of any kernel that streams W. */
+int dm_debug_read_stream(dm_ctx* ctx, const void* ptr, size_t bytes, void* stream);
+
 /* Reads and clears the context's device error word (0 = none); synchronises `stream` first.
  * Non-zero means a kernel abandoned an internal wait and the outputs of that call are invalid. */
 int dm_device_error(dm_ctx* ctx, void* stream, uint32_t* out_code);

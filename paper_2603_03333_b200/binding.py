@@ -48,6 +48,7 @@ SIGNATURES = {
                                          _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_debug_masks": (_ci, [_vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
+    "dm_debug_read_stream": (_ci, [_vp, _vp, ctypes.c_size_t, _vp]),
     "dm_device_error": (_ci, [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]),
     "dm_profile_head": (_ci, [_vp, _ci]),
     "dm_profile_read": (_ci, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_ci)]),
@@ -326,6 +327,11 @@ class Context:
         _check(lib().dm_debug_masks(self._h, B, T, K, d, p, seed, seq_base, _ptr(out), _stream(self.device)),
                "dm_debug_masks")
         return out
+
+    def debug_read_stream(self, t: torch.Tensor):
+        """One read-only pass over a CUDA tensor's bytes (for measuring the read-only HBM rate)."""
+        _check(lib().dm_debug_read_stream(self._h, _ptr(t), t.numel() * t.element_size(), _stream(self.device)),
+               "dm_debug_read_stream")
 
     def device_error(self) -> int:
         code = ctypes.c_uint32()

@@ -164,9 +164,9 @@ int dm_create(dm_ctx** out, int device) {
     dm_ctx* c = new (std::nothrow) dm_ctx();
     if (c == nullptr) return DM_ECUDA;
     c->device = device;
-    // two words: the device error word, then the finished-CTA ticket of the fused kernel
-    if (cudaMalloc(&c->err, 2 * sizeof(uint32_t)) != cudaSuccess ||
-        cudaMemset(c->err, 0, 2 * sizeof(uint32_t)) != cudaSuccess) {
+    // the device error word, the finished-CTA ticket of the fused kernel, a sink for dm_debug_read_stream
+    if (cudaMalloc(&c->err, 4 * sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(c->err, 0, 4 * sizeof(uint32_t)) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(c->err);
         delete c;
@@ -554,6 +554,16 @@ int dm_debug_masks(dm_ctx* c, int B, int T, int K, int d, float p, uint64_t seed
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
     return launch_debug_masks(B, T, K, d, mk, (uint32_t)seq_base, c->mask_mode, out_bits, static_cast<cudaStream_t>(stream));
+}
+
+int dm_debug_read_stream(dm_ctx* c, const void* ptr, size_t bytes, void* stream) {
+    if (c == nullptr || ptr == nullptr || bytes < 16 || (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) return DM_ECUDA;
+    // the sink is the ticket word's neighbour: it is only ever written with a value nobody reads
+    return launch_read_stream(ptr, bytes, c->err + 2, sms, static_cast<cudaStream_t>(stream));
 }
 
 int dm_device_error(dm_ctx* c, void* stream, uint32_t* out_code) {

@@ -60,6 +60,27 @@ int launch_finalize(const unsigned long long* partials, int n_slices, int rows,
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 
+// Measurement aid: a plain read-only stream over a buffer (16-byte loads, grid-stride, XOR-folded
+// so that the loads cannot be dropped).  Its rate is the read-only HBM ceiling of the part.
+__global__ void __launch_bounds__(1024, 2)
+read_stream_kernel(const uint4* __restrict__ p, size_t n16, unsigned int* __restrict__ sink) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    unsigned int acc = 0;
+    for (; i + 3 * stride < n16; i += 4 * stride) {
+        const uint4 a = __ldcs(p + i), b = __ldcs(p + i + stride), c = __ldcs(p + i + 2 * stride),
+                    e = __ldcs(p + i + 3 * stride);
+        acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ e.x ^ e.y ^ e.z ^ e.w;
+    }
+    for (; i < n16; i += stride) { const uint4 a = __ldcs(p + i); acc ^= a.x ^ a.y ^ a.z ^ a.w; }
+    if (acc == 0x9E3779B9u) atomicExch(sink, acc);   // practically never: keeps the loads alive
+}
+
+int launch_read_stream(const void* ptr, size_t bytes, unsigned int* sink, int sms, cudaStream_t stream) {
+    read_stream_kernel<<<sms * 4, 1024, 0, stream>>>(static_cast<const uint4*>(ptr), bytes / 16, sink);
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+}
+
 // Eq. 1 keep bits, one 32-bit word (eight Philox quads) per thread.
 __global__ void debug_masks_kernel(int n_paths, int K, int T, int d, MaskKey mk, uint32_t seq_base_lo, int shared_masks,
                                    uint32_t* __restrict__ out_bits) {

@@ -74,6 +74,8 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidd
                  const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
                  unsigned long long* best = nullptr, bool* folded_out = nullptr);
 
+int launch_read_stream(const void* ptr, size_t bytes, unsigned int* sink, int sms, cudaStream_t stream);
+
 // JS-divergence acceptance (Eq. 4, Eq. 5, Algorithm 1) on logits [B*T*K][V] written by a head kernel.
 int js_chunks(int V);
 size_t js_workspace_floats(int V, int max_rows, int max_hidden);
