@@ -51,6 +51,8 @@ CONFIGS = {
     "llama70b": Config("llama70b", d=8192, V=128256, dtype=BF16, B=16, T=8, K=16, p=0.1),
     # the Llama-3-8B head at the upper end of the HBM-bound range (256 paths: staged operand, CTA pairs)
     "llama8b_k32": Config("llama8b_k32", d=4096, V=128256, dtype=BF16, B=1, T=8, K=32, p=0.1),
+    # ... and a tensor-bound call on the same head (512 paths: two row blocks per launch)
+    "llama8b_b2k32": Config("llama8b_b2k32", d=4096, V=128256, dtype=BF16, B=2, T=8, K=32, p=0.1),
 }
 
 
