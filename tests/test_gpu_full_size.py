@@ -117,3 +117,27 @@ def test_llama70b_config_sampled():
         _check_sampled_paths(ctx, cfg, work, got["tokens"], paths)
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("name,reps", [("llama8b", 300), ("llama8b_k32", 100), ("llama8b_b2k32", 60)])
+def test_full_size_runs_are_deterministic(name, reps):
+    """The same call repeated back to back (one launch; CTA pairs; two row blocks per launch) must
+    give the same bytes every time, also when other seeds run in between: a missed barrier or a
+    stale partial would show up here long before it shows up in a parity sample."""
+    cfg = wl.CONFIGS[name]
+    work = wl.make_workload(cfg, device=DEV)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+        first = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
+        scratch = ctx.alloc_outputs(cfg.B, cfg.T, cfg.K)
+        for n in range(reps):
+            ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED + 1 + n, out=scratch)   # another seed in between
+            again = ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED)
+            if n % 20 == 19 or n == reps - 1:
+                got = to_np(again)
+                for key in first:
+                    assert np.array_equal(first[key], got[key]), (n, key)
+        assert ctx.device_error() == 0
+    finally:
+        ctx.close()
