@@ -74,9 +74,10 @@ int dm_destroy(dm_ctx* ctx);
  * next dm_set_head.  Reserves workspace for calls of up to `max_rows` rows (rows = B*T*K, or
  * B*N_h*K for trees) and `max_hidden_rows` = rows/K hidden rows (used only by the *_host entry
  * point's staging buffers).  Requirements: V >= 1; d >= 4 and d % 4 == 0 (fp32) or d % 8 == 0
- * (bf16), else DM_EUNSUPPORTED; heads that run on the CUDA-core kernel also need one hidden row to
- * fit 200 KB of shared memory (d <= 51200 fp32, 102400 bf16), which verify calls report.  bf16 heads with d % 64 == 0 run on the tcgen05 tensor-core
- * kernel, everything else on the CUDA-core kernel.  Synchronises the device (re-allocation). */
+ * (bf16), else DM_EUNSUPPORTED.  bf16 heads with d % 64 == 0 run on the tcgen05 tensor-core
+ * kernel, everything else on the CUDA-core kernel, which also needs one hidden row to fit
+ * 200 KB of shared memory (d <= 51200 fp32, 102400 bf16; verify calls report DM_EUNSUPPORTED
+ * beyond).  Synchronises the device (re-allocation); pins host memory for the *_host call. */
 int dm_set_head(dm_ctx* ctx, const void* W, int V, int d, int dtype, int max_rows, int max_hidden_rows);
 
 /* Force a kernel family (DM_IMPL_*) for later calls; DM_IMPL_AUTO restores the default choice.
