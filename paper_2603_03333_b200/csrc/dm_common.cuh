@@ -66,8 +66,10 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1
     constexpr uint32_t WA = 0x9E3779B9u, WB = 0xBB67AE85u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        uint32_t hi_a = __umulhi(MA, c.x), lo_a = MA * c.x;
-        uint32_t hi_b = __umulhi(MB, c.z), lo_b = MB * c.z;
+        // one widening multiply per product (both halves from a single 32x32->64 instruction)
+        const unsigned long long pa = (unsigned long long)MA * c.x, pb = (unsigned long long)MB * c.z;
+        const uint32_t hi_a = (uint32_t)(pa >> 32), lo_a = (uint32_t)pa;
+        const uint32_t hi_b = (uint32_t)(pb >> 32), lo_b = (uint32_t)pb;
         c = make_uint4(hi_b ^ c.y ^ k0, lo_b, hi_a ^ c.w ^ k1, lo_a);
         k0 += WA;
         k1 += WB;
