@@ -283,6 +283,55 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+SWEEPS = {
+    # (head name, V, d, [(B, T, K), ...]): the row counts of the tables in the design notes
+    "llama8b": (128256, 4096, [(1, 1, 8), (1, 2, 8), (1, 5, 8), (1, 8, 8), (1, 5, 16), (1, 8, 16), (1, 5, 32),
+                               (1, 8, 32), (3, 5, 20), (4, 8, 16), (8, 8, 16)]),
+    "qwen8b": (151936, 4096, [(B, 7, K) for B in (1, 8, 32) for K in (4, 8, 16, 32)]),
+    "llama70b": (128256, 8192, [(1, 8, 16), (16, 8, 16)]),
+}
+
+
+def run_sweep(args):
+    """Not the benchmark line: times the head kernel(s) and the whole call over a list of call
+    sizes on one head and prints one JSON line per size (fractions against the measured peaks)."""
+    import torch
+    import paper_2603_03333_b200 as pk
+    from paper_2603_03333_b200 import workloads as wl
+    V, d, cases = SWEEPS[args.sweep]
+    dev, peaks = "cuda:0", load_peaks()
+    W = wl.make_head(V, d, wl.BF16, seed=1, device=dev)
+    ctx = pk.Context(0)
+    ctx.set_head(W, max_rows=max(B * T * K for B, T, K in cases), max_hidden_rows=max(B * T for B, T, K in cases))
+    for B, T, K in cases:
+        H = wl.make_hidden(B * T, d, wl.BF16, seed=2, device=dev).view(B, T, d)
+        draft = torch.zeros((B, T), dtype=torch.int32, device=dev)
+        out = ctx.alloc_outputs(B, T, K)
+        rows, reps = B * T * K, (50 if B * T * K <= 512 else 8)
+        for i in range(5):
+            ctx.verify_batched(H, draft, K, 0.1, 1 + i, out=out)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            ctx.verify_batched(H, draft, K, 0.1, 100 + i, out=out)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx.profile_head(True)
+        for i in range(reps):
+            ctx.verify_batched(H, draft, K, 0.1, 100 + i, out=out)
+        torch.cuda.synchronize()
+        ms, n = ctx.profile_read()
+        ctx.profile_head(False)
+        t_head, t_call = ms / n * 1e-3, e0.elapsed_time(e1) / reps * 1e-3
+        t_mem = (V * d + B * T * d) * 2 / (peaks["hbm_gbs"] * 1e9)
+        t_flop = 2.0 * rows * V * d / (peaks["bf16_tflops"] * 1e12)
+        print(json.dumps(dict(head=args.sweep, B=B, T=T, K=K, rows=rows, head_us=round(t_head * 1e6, 1),
+                              call_us=round(t_call * 1e6, 1), bound="hbm" if t_mem >= t_flop else "tensor",
+                              frac=round(max(t_mem, t_flop) / t_head, 3), launches=ctx.last_launches())), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -291,9 +340,12 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default=None, choices=sorted(SWEEPS), help="time a list of call sizes on one head")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)
