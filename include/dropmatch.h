@@ -71,7 +71,10 @@ int dm_destroy(dm_ctx* ctx);
 
 /* Describe the LM head (Eq. 3): W is a device pointer to V*d elements, row-major [V,d],
  * 16-byte aligned, caller-owned; it is read, never written, by every verify call until the
- * next dm_set_head.  Reserves workspace for calls of up to `max_rows` rows (rows = B*T*K, or
+ * next dm_set_head, and it must be complete before a call is enqueued: the tensor-core kernel
+ * is launched with programmatic stream serialization and starts streaming W while the kernel
+ * ahead of it in the stream is still finishing (H, the drafts and all outputs are only touched
+ * after that kernel has completed).  Reserves workspace for calls of up to `max_rows` rows (rows = B*T*K, or
  * B*N_h*K for trees) and `max_hidden_rows` = rows/K hidden rows (used only by the *_host entry
  * point's staging buffers).  Requirements: V >= 1; d >= 4 and d % 4 == 0 (fp32) or d % 8 == 0
  * (bf16), else DM_EUNSUPPORTED.  bf16 heads with d % 64 == 0 run on the tcgen05 tensor-core

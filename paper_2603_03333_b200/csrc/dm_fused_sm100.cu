@@ -73,6 +73,7 @@ struct FusedParams {
     int n_slots;      // accumulator slots in TMEM (512 / n_pad)
     int nsw, nsb;     // stages of the W ring and of the operand ring
     int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
+    int pdl;          // launched with programmatic stream serialization: see the griddep_wait() calls
     int row_blocks;   // 1, or 2: two blocks of 256 paths share one pass over W (see fused_launch)
     RowMap map;
     uint32_t key0, key1, thr;
@@ -172,6 +173,11 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     if (kPair) ptx::cluster_sync_all();   // the other CTA's barriers are initialised before anyone signals them
     ptx::tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
+    // The next call's kernel may be scheduled as soon as SMs free up: its prologue and its first W
+    // loads then overlap this kernel's tail.  W is never written while calls are in flight, so the
+    // W producer and the MMA issuer need not wait for the kernel ahead; whoever reads H or the
+    // staged operand, or writes global memory, does (griddep_wait below).
+    if (P.pdl) ptx::griddep_launch_dependents();
 
     const int v_cta0 = slice * P.slice_rows;
     int my_tiles = 0;
@@ -289,6 +295,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             // The masked rows were written to the staging buffer by mask_operand_kernel; one
             // thread streams the [n_pad x 64] block of every (group, block) step through TMA.
             if (threadIdx.x != (kFirstExpWarp + 4) * 32) return;
+            if (P.pdl) ptx::griddep_wait();   // the staged operand is written by the kernel ahead
             const int b_rows = kPair ? P.n_pad / 2 : P.n_pad;      // a pair splits the operand rows
             const int b_row0 = row0 + (int)rank * b_rows;
             const uint32_t b_stage_bytes = (uint32_t)b_rows * (kBlockK * 2);
@@ -314,6 +321,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         }
     } else if (warp >= kFirstExpWarp) {
         // ------------------------------------------------------------------ operand builders
+        if (P.pdl) ptx::griddep_wait();       // H may be the output of the kernel ahead
         const int e = warp - kFirstExpWarp;
         const int grp = e % P.nsb, sub = e / P.nsb;
         const uint32_t b_stage_bytes = (uint32_t)P.n_pad * (kBlockK * 2);
@@ -393,6 +401,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // ------------------------------------------------------------------ epilogue
         // Warps 2-5, plus warps 6-9 in staged mode, where no operand is built.  Warp w reads TMEM
         // lanes 32*(w mod 4)..+31; the warps of a lane quarter share the column chunks.
+        if (P.pdl) ptx::griddep_wait();       // global writes (and the shared per-row best) only after the kernel ahead
         const int ew = warp & 3;                      // lane quarter = row of s_best
         const int set = warp < kFirstExpWarp ? 0 : 1;
         const int n_sets = P.staged ? 2 : 1;
@@ -854,25 +863,35 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.ticket = ticket;
         P.best = best;
         if (P.fold) { P.fin = *fin; if (folded_out) *folded_out = true; }
-        if (plan.pair) {
-            cudaLaunchConfig_t cfg{};   // clusters of two CTAs
-            cfg.gridDim = dim3((unsigned)grid);
-            cfg.blockDim = dim3(kThreads);
-            cfg.dynamicSmemBytes = plan.total;
-            cfg.stream = stream;
-            cudaLaunchAttribute attr{};
-            attr.id = cudaLaunchAttributeClusterDimension;
-            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-            cfg.attrs = &attr;
-            cfg.numAttrs = 1;
-            if (cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, geo.tmap_w, fs->tmap_b[P.n_pad / 32 - 1], P) !=
-                cudaSuccess) {
-                cudaGetLastError();
-                return DM_ECUDA;
-            }
-        } else {
-            fused_head_kernel<false><<<grid, kThreads, plan.total, stream>>>(
-                geo.tmap_w, plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : geo.tmap_w, P);
+        // Programmatic stream serialization, except when the row selection of the debug call could
+        // itself be the output of the kernel ahead (it is read in the prologue).
+        P.pdl = map.sel == nullptr ? 1 : 0;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = plan.total;
+        cfg.stream = stream;
+        cudaLaunchAttribute attrs[2]{};
+        int n_attrs = 0;
+        if (P.pdl) {
+            attrs[n_attrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attrs[n_attrs].val.programmaticStreamSerializationAllowed = 1;
+            ++n_attrs;
+        }
+        if (plan.pair) {   // clusters of two CTAs
+            attrs[n_attrs].id = cudaLaunchAttributeClusterDimension;
+            attrs[n_attrs].val.clusterDim.x = 2; attrs[n_attrs].val.clusterDim.y = 1; attrs[n_attrs].val.clusterDim.z = 1;
+            ++n_attrs;
+        }
+        cfg.attrs = attrs;
+        cfg.numAttrs = n_attrs;
+        const cudaError_t launched =
+            plan.pair ? cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, geo.tmap_w, fs->tmap_b[P.n_pad / 32 - 1], P)
+                      : cudaLaunchKernelEx(&cfg, fused_head_kernel<false>, geo.tmap_w,
+                                           plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : geo.tmap_w, P);
+        if (launched != cudaSuccess) {
+            cudaGetLastError();
+            return DM_ECUDA;
         }
         if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
         ++launches;

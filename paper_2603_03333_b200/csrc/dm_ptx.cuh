@@ -178,6 +178,18 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint16_t cta_mask)
                  ::"r"(bar), "h"(cta_mask) : "memory");
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// A kernel launched with programmatic stream serialization may start before the kernel ahead of
+// it in the stream has finished.  griddep_wait() returns once that kernel has completed and its
+// writes are visible: everything before it must not touch what that kernel produces.
+// griddep_launch_dependents() tells the runtime that the next such kernel may be scheduled.
+__device__ __forceinline__ void griddep_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // Named barrier among a subset of warps.
 __device__ __forceinline__ void bar_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
