@@ -27,7 +27,7 @@ WORKLOAD = "llama8b"   # Llama-3-8B-shaped head: the configuration the metric is
 
 # DRAM bytes (read + write) of one fused head-kernel launch on this workload, from the ncu capture
 # summarised in profiles/; None until a capture exists.
-NCU_TRAFFIC_BYTES = {"llama8b": 1050957000 + 3879000, "llama8b_k32": 1059198000 + 4144000}
+NCU_TRAFFIC_BYTES = {"llama8b": 1051084000 + 4251000, "llama8b_k32": 1059248000 + 5305000}
 
 
 def load_peaks():
