@@ -73,6 +73,7 @@ SMALL = [
     wl.Config("js_bf16_staged", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1),   # staged operand, CTA pairs
     wl.Config("js_f32", d=100, V=517, dtype=wl.F32, B=2, T=3, K=7, p=0.2, draft_mode="toy"),   # CUDA-core family
     wl.Config("js_k1", d=256, V=700, dtype=wl.BF16, B=1, T=2, K=1, p=0.2),
+    wl.Config("js_rows288", d=128, V=40000, dtype=wl.BF16, B=3, T=6, K=16, p=0.1),       # two head launches with logits
     wl.Config("js_k24", d=128, V=5000, dtype=wl.BF16, B=1, T=3, K=24, p=0.2),            # 17..32 paths in registers
     wl.Config("js_k40", d=128, V=2000, dtype=wl.BF16, B=1, T=2, K=40, p=0.2),            # more than fit: series by series
 ]
