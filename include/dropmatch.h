@@ -161,7 +161,8 @@ int dm_enable_js(dm_ctx* ctx, int max_rows, int max_hidden_rows);
  *   out_js[B,T,K+1]     device, fp32: JS(p^(i) || pbar) for i < K, then JS(phat || pbar)
  *   out_js_ok[B,T]      device, 1 iff Eq. 5 holds (may be NULL)
  *   the rest            as for dropmatch_verify_batched
- * Needs dm_enable_js with room for the call, else DM_EWORKSPACE.  Only enqueues work. */
+ * Needs dm_enable_js with room for the call, else DM_EWORKSPACE; B*T <= 65535, else
+ * DM_EUNSUPPORTED (checked before anything is launched).  Only enqueues work. */
 int dropmatch_verify_js(dm_ctx* ctx, const void* H, const int32_t* draft, const float* draft_prob, int B, int T,
                         int K, float p, uint64_t seed, uint64_t seq_base, int32_t* out_tokens,
                         int32_t* out_counts, float* out_js, int32_t* out_js_ok, int32_t* out_accept_len,
@@ -254,14 +255,32 @@ int dm_debug_logits(dm_ctx* ctx, const void* H, int B, int T, const int32_t* row
 int dm_debug_masks(dm_ctx* ctx, int B, int T, int K, int d, float p, uint64_t seed,
                    uint64_t seq_base, uint32_t* out_bits, void* stream);
 
+/* Debug: the masked hidden rows themselves (Eq. 1 and Eq. 2 without the 1/(1-p) factor), exactly
+ * as the tensor-core kernel stages them for calls of more than 64 paths or so: out[B*T*K, d] in
+ * the head's storage type, row (b*T+t)*K+i = H[b,t,:] with the dropped elements set to zero.
+ * bf16 heads only (DM_EUNSUPPORTED otherwise); out is a device pointer, 16-byte aligned. */
+int dm_debug_masked_operand(dm_ctx* ctx, const void* H, int B, int T, int K, float p, uint64_t seed,
+                            uint64_t seq_base, void* out, void* stream);
+
 /* Measurement aid: enqueues one read-only pass over `bytes` bytes at device pointer `ptr` (16-byte
  * aligned; the bytes beyond a multiple of 16 are not read).  Timed over a buffer much larger than
  * L2 it gives the read-only HBM rate of the part, the ceiling of any kernel that streams W. */
 int dm_debug_read_stream(dm_ctx* ctx, const void* ptr, size_t bytes, void* stream);
 
 /* Reads and clears the context's device error word (0 = none); synchronises `stream` first.
- * Non-zero means a kernel abandoned an internal wait and the outputs of that call are invalid. */
+ * Non-zero means a kernel abandoned an internal wait.  The outputs of that call, and of every
+ * later call until this function has cleared the word, are then the fail-safe values written on
+ * the device, so that no consumer further down the stream mistakes them for results:
+ * tokens -1, counts and hits 0, accepted length 0, best node -1, node_ok 0, plain/next tokens -1
+ * (the left-to-right rule of Sec. 2 with nothing accepted). */
 int dm_device_error(dm_ctx* ctx, void* stream, uint32_t* out_code);
+
+/* Debug: how many clock cycles a kernel of this context waits on one of its internal barriers
+ * before it gives up, sets the device error word and winds down (0 restores the default, about
+ * one second; the time a call spends queued behind the kernel ahead of it counts).  A limit of
+ * a few cycles makes the first wait that is not satisfied at once run out: the tests use that
+ * to exercise the wind-down and the fail-safe outputs without hanging or faulting anything. */
+int dm_debug_set_wait_limit(dm_ctx* ctx, uint64_t cycles);
 
 /* Timing of the head kernel alone (the dominant kernel).  While enabled, every verify call
  * records a CUDA event on `stream` before and after its masked-head kernel launch(es) (not

@@ -48,8 +48,10 @@ SIGNATURES = {
                                          _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dm_debug_logits": (_ci, [_vp, _vp, _ci, _ci, _vp, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_debug_masks": (_ci, [_vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
+    "dm_debug_masked_operand": (_ci, [_vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
     "dm_debug_read_stream": (_ci, [_vp, _vp, ctypes.c_size_t, _vp]),
     "dm_device_error": (_ci, [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]),
+    "dm_debug_set_wait_limit": (_ci, [_vp, _u64]),
     "dm_profile_head": (_ci, [_vp, _ci]),
     "dm_profile_read": (_ci, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_ci)]),
     "dm_workspace_bytes": (ctypes.c_size_t, [_vp]),
@@ -328,6 +330,15 @@ class Context:
                "dm_debug_masks")
         return out
 
+    def debug_masked_operand(self, H, K, p, seed, seq_base=0):
+        """-> [B*T*K, d] tensor of the head's dtype: every path's hidden row with its dropped elements zeroed."""
+        B, T, d = H.shape
+        _dev(H, self._tdtype(), "H")
+        out = torch.empty((B * T * K, d), dtype=H.dtype, device=self.device)
+        _check(lib().dm_debug_masked_operand(self._h, _ptr(H), B, T, K, p, seed, seq_base, _ptr(out),
+                                             _stream(self.device)), "dm_debug_masked_operand")
+        return out
+
     def debug_read_stream(self, t: torch.Tensor):
         """One read-only pass over a CUDA tensor's bytes (for measuring the read-only HBM rate)."""
         _check(lib().dm_debug_read_stream(self._h, _ptr(t), t.numel() * t.element_size(), _stream(self.device)),
@@ -337,6 +348,9 @@ class Context:
         code = ctypes.c_uint32()
         _check(lib().dm_device_error(self._h, _stream(self.device), ctypes.byref(code)), "dm_device_error")
         return code.value
+
+    def debug_set_wait_limit(self, cycles: int):
+        _check(lib().dm_debug_set_wait_limit(self._h, cycles), "dm_debug_set_wait_limit")
 
     def profile_head(self, enable: bool):
         _check(lib().dm_profile_head(self._h, int(enable)), "dm_profile_head")

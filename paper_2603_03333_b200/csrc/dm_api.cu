@@ -15,6 +15,7 @@ struct dm_ctx {
     int max_rows = 0, max_hidden = 0;
     int impl = DM_IMPL_AUTO;
     int mask_mode = DM_MASK_PER_POSITION;
+    long long wait_limit = 0;                // clock cycles a kernel waits on a barrier before it gives up; 0 = default
     int last_impl = 0, last_launches = 0;
     // workspace (device)
     unsigned long long* partials = nullptr;  // [kMaxSlices][max_rows]
@@ -94,7 +95,9 @@ int pick_impl(const dm_ctx* c, int rows, int* impl) {
 
 // Masked head + per-slice argmax for `rows` rows, then merge/histogram/acceptance.
 int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const MaskKey& mk,
-               const FinalizeArgs& fa, cudaStream_t stream, float* logits_out = nullptr) {
+               const FinalizeArgs& fa_in, cudaStream_t stream, float* logits_out = nullptr) {
+    FinalizeArgs fa = fa_in;
+    fa.err = c->err;   // results are replaced by "nothing accepted" if a kernel of the call gives up on a wait
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
     if (rows > c->max_rows) return DM_EWORKSPACE;
     if (finalize_smem_bytes(fa.T, fa.K + fa.plain, fa.N) > 200 * 1024) return DM_EUNSUPPORTED;
@@ -117,7 +120,7 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
                           logits_out, c->err, stream, &launches, &fa, c->err + 1,
-                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded);
+                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded, nullptr, c->wait_limit);
     else {
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, logits_out, c->err, stream);
         launches = 1;
@@ -263,16 +266,28 @@ int dropmatch_partial_best(dm_ctx* c, const void* H, int B, int T, int K, float 
     st = pick_impl(c, rows, &impl);
     if (st != DM_OK) return st;
     int n_slices = 0, launches = 1;
-    if (impl == DM_IMPL_TCGEN05)   // no finalize arguments: the kernels leave per-slice partials
+    bool reduced = false;
+    unsigned long long* out = reinterpret_cast<unsigned long long*>(out_packed);
+    if (impl == DM_IMPL_TCGEN05) {
+        // A call of one launch: the CTAs reduce straight into the caller's array (zero first), no
+        // second kernel.  Larger calls leave per-slice partials that a small kernel merges.
+        if (cudaMemsetAsync(out, 0, (size_t)rows * sizeof(unsigned long long), s) != cudaSuccess) {
+            cudaGetLastError();
+            return DM_ECUDA;
+        }
         st = fused_launch(c->fused, c->head, H, B * T, rows, map, mk, &n_slices, c->partials, nullptr, c->err, s,
-                          &launches);
-    else
+                          &launches, nullptr, nullptr, nullptr, &reduced, out, c->wait_limit);
+    } else {
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, s);
+    }
     if (st != DM_OK) return st;
-    st = launch_merge_partials(c->partials, n_slices, rows, reinterpret_cast<unsigned long long*>(out_packed), s);
-    if (st != DM_OK) return st;
+    if (!reduced) {
+        st = launch_merge_partials(c->partials, n_slices, rows, out, s);
+        if (st != DM_OK) return st;
+        ++launches;
+    }
     c->last_impl = impl;
-    c->last_launches = launches + 1;
+    c->last_launches = launches;
     return DM_OK;
 }
 
@@ -292,8 +307,15 @@ int dropmatch_finalize_packed(dm_ctx* c, const uint64_t* packed, int n_parts, co
     fa.draft = draft; fa.out_hits = out_draft_hits;
     fa.N = 0;
     fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    fa.err = c->err;
     return launch_finalize(reinterpret_cast<const unsigned long long*>(packed), n_parts, B * T * K, fa,
                            static_cast<cudaStream_t>(stream));
+}
+
+int dm_debug_set_wait_limit(dm_ctx* c, uint64_t cycles) {
+    if (c == nullptr || cycles > (1ull << 40)) return DM_EINVAL;
+    c->wait_limit = (long long)cycles;
+    return DM_OK;
 }
 
 int dm_set_mask_mode(dm_ctx* c, int mode) {
@@ -440,6 +462,7 @@ int dropmatch_verify_js(dm_ctx* c, const void* H, const int32_t* draft, const fl
         out_js == nullptr || out_accept_len == nullptr)
         return DM_EINVAL;
     const long long hidden = (long long)B * T, rows = hidden * K;
+    if (hidden > kJsMaxPositions) return DM_EUNSUPPORTED;   // before anything is launched or overwritten
     if (c->js_logits == nullptr || rows > c->js_max_rows || hidden > c->js_max_hidden) return DM_EWORKSPACE;
     MaskKey mk;
     if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
@@ -457,7 +480,7 @@ int dropmatch_verify_js(dm_ctx* c, const void* H, const int32_t* draft, const fl
     st = run_verify(c, H, (int)rows, map, mk, fa, s, c->js_logits);
     if (st != DM_OK) return st;
     st = launch_js(c->js_logits, draft_prob, c->js_ws, c->head.V, B, T, K, out_tokens, draft, out_js, out_js_ok,
-                   out_accept_len, s);
+                   out_accept_len, c->err, s);
     if (st != DM_OK) return st;
     c->last_launches += 3;
     return DM_OK;
@@ -554,6 +577,19 @@ int dm_debug_masks(dm_ctx* c, int B, int T, int K, int d, float p, uint64_t seed
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
     return launch_debug_masks(B, T, K, d, mk, (uint32_t)seq_base, c->mask_mode, out_bits, static_cast<cudaStream_t>(stream));
+}
+
+int dm_debug_masked_operand(dm_ctx* c, const void* H, int B, int T, int K, float p, uint64_t seed,
+                            uint64_t seq_base, void* out, void* stream) {
+    int st = check_common(c, H, B, T, K);
+    if (st != DM_OK) return st;
+    if (out == nullptr || (reinterpret_cast<uintptr_t>(out) & 15u) != 0) return DM_EINVAL;
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};
+    return fused_debug_operand(c->head, H, B * T * K, map, mk, out, c->err, static_cast<cudaStream_t>(stream));
 }
 
 int dm_debug_read_stream(dm_ctx* c, const void* ptr, size_t bytes, void* stream) {

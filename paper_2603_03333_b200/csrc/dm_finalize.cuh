@@ -52,6 +52,28 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
     int32_t* flag = sm + TK;       // chain: ok[T]; tree: test[N] then ok/depth packed [N]
     const size_t row0 = (size_t)b * TK;
     const size_t out0 = (size_t)b * a.T * a.K;
+    // A kernel of this call gave up on a wait (device error word set): the partial maxima are
+    // incomplete.  Nothing may then look accepted to a consumer further down the stream: no token
+    // (-1), empty histogram, accepted length 0 (the left-to-right rule rejects everything).
+    if (a.err != nullptr && *reinterpret_cast<const volatile uint32_t*>(a.err) != 0u) {
+        for (int x = tid; x < a.T * a.K; x += nthreads) { a.out_tokens[out0 + x] = -1; a.out_counts[out0 + x] = 0; }
+        for (int t = tid; t < a.T; t += nthreads)
+            if (a.out_plain) a.out_plain[(size_t)b * a.T + t] = -1;
+        if (a.N == 0) {
+            for (int t = tid; t < Td; t += nthreads)
+                if (a.out_hits) a.out_hits[(size_t)b * Td + t] = 0;
+        } else {
+            for (int n = tid; n < a.N; n += nthreads)
+                if (a.out_node_ok) a.out_node_ok[(size_t)b * a.N + n] = 0;
+        }
+        if (tid == 0) {
+            a.out_accept_len[b] = 0;
+            if (a.N > 0) a.out_best_node[b] = -1;
+            if (a.out_next) a.out_next[b] = -1;
+        }
+        sync();
+        return;
+    }
     auto store_token = [&](int x, int32_t tok) {
         toks[x] = tok;
         const int t = x / Kp, i = x - t * Kp;

@@ -49,7 +49,7 @@ constexpr int kMaxNPad = 256;               // UMMA N limit
 constexpr int kWStageBytes = kTileM * kBlockK * 2;
 constexpr int kTmemCols = 512;
 constexpr int kMaxWStages = 12;
-constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
+constexpr long long kWaitLimitCycles = 2000000000ll;   // default limit of every wait: about one second
 constexpr int kPollNs = 32;                 // pause between polls of a barrier on the critical path
 constexpr int kIdlePollNs = 500;            // ... and of one that completes once per tile group
 constexpr int kSmemLimit = 227 * 1024;
@@ -74,6 +74,7 @@ struct FusedParams {
     int nsw, nsb;     // stages of the W ring and of the operand ring
     int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
     int pdl;          // launched with programmatic stream serialization: see the griddep_wait() calls
+    long long wait_limit;   // clock cycles after which a wait on an mbarrier gives up (see dm_debug_set_wait_limit)
     int row_blocks;   // 1, or 2: two blocks of 256 paths share one pass over W (see fused_launch)
     RowMap map;
     uint32_t key0, key1, thr;
@@ -81,8 +82,10 @@ struct FusedParams {
     unsigned long long* partials;   // [vocabulary slice][rows_total]
     float* dbg_logits;              // [rows_total][V] or null
     uint32_t* err;
-    // When `fold` is set the last CTA to finish also merges the partials and runs the histogram
-    // and the acceptance (a call of one launch): `ticket` counts finished CTAs and is left at 0.
+    // fold != 0 (a call of one launch): the CTAs reduce their per-path best into `best` with atomic
+    // maxima instead of writing per-slice partials.  fold == 1: the last CTA to finish also runs the
+    // histogram and the acceptance and zeroes `best` again; `ticket` counts finished CTAs and is
+    // left at 0.  fold == 2: `best` is the caller's array (zero before the launch), nothing more.
     int fold;
     unsigned int* ticket;
     unsigned long long* best;       // [rows_total], all zero between calls: CTAs reduce into it when folding
@@ -126,6 +129,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_bar + n_bars);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
     volatile unsigned int* s_ticket = reinterpret_cast<volatile unsigned int*>(s_tmem + 2);
+    volatile int* s_never = reinterpret_cast<volatile int*>(s_tmem + 3);   // stays 0: for the one wait that an abort must not cut short
 
     const int wps = kExpWarps / P.nsb;   // operand-builder warps per ring stage
     const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;   // 0 = leader of the pair
@@ -150,6 +154,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, kPair ? 16 : P.staged ? 8 : 4); }
         ptx::mbar_init(dealloc_bar, 1);
         *s_abort = 0;
+        *s_never = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
     }
@@ -208,7 +213,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
                 int v_tile = v_first;
                 for (int tile = t0; tile < t1; ++tile, v_tile += P.tile_rows) {
-                    if (!ptx::mbar_wait<kPollNs>(bar_empty, empty_parity, s_abort, kWaitLimitCycles)) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_empty, empty_parity, s_abort, P.wait_limit)) {
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                         return;
                     }
@@ -245,7 +250,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             const int t0 = g * G, t1 = min(my_tiles, t0 + G);
             const int slot0 = slot;
             for (int tile = t0; tile < t1; ++tile) {   // the group's accumulator slots must be drained
-                if (!ptx::mbar_wait<kPollNs>(slot_empty + 8 * slot, slot_parity, s_abort, kWaitLimitCycles)) {
+                if (!ptx::mbar_wait<kPollNs>(slot_empty + 8 * slot, slot_parity, s_abort, P.wait_limit)) {
                     atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
                     return;
                 }
@@ -253,14 +258,14 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             }
             ptx::tc_fence_after();
             for (int kb = 0; kb < P.kb_count; ++kb) {
-                if (!ptx::mbar_wait<kPollNs>(bar_br, b_parity, s_abort, kWaitLimitCycles)) {
+                if (!ptx::mbar_wait<kPollNs>(bar_br, b_parity, s_abort, P.wait_limit)) {
                     atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
                     return;
                 }
                 int sl = slot0;
                 uint32_t d_tmem = tmem_base + (uint32_t)(slot0 * P.n_pad);
                 for (int tile = t0; tile < t1; ++tile) {
-                    if (!ptx::mbar_wait<kPollNs>(bar_wf, w_parity, s_abort, kWaitLimitCycles)) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_wf, w_parity, s_abort, P.wait_limit)) {
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
                         return;
                     }
@@ -303,7 +308,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             int stage = 0;
             for (int g = 0; g < n_groups; ++g)
                 for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
-                    if (!ptx::mbar_wait<kPollNs>(bar_e, parity, s_abort, kWaitLimitCycles)) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_e, parity, s_abort, P.wait_limit)) {
                         atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                         return;
                     }
@@ -352,7 +357,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                 }
             }
             if (!ptx::mbar_wait_warp<kPollNs>(b_empty + 8 * grp, ((m / P.nsb) & 1) ^ 1, s_abort,
-                                              kWaitLimitCycles)) {
+                                              P.wait_limit)) {
                 atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
                 break;
             }
@@ -424,7 +429,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             for (int tile = t0; tile < t1; ++tile) {
                 // the tcgen05.ld below needs the whole warp: the outcome of the wait is warp-uniform
                 if (!ptx::mbar_wait_warp<kIdlePollNs>(slot_full + 8 * (tile % P.n_slots), (tile / P.n_slots) & 1,
-                                                      s_abort, kWaitLimitCycles)) {
+                                                      s_abort, P.wait_limit)) {
                     atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_FULL);
                     alive = false;
                     break;
@@ -536,9 +541,13 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         }
         // ------------------------------------------------------------------ teardown
         // Every accumulator has been read, hence every MMA and every TMA load has completed.
-        // After an abandoned wait, give copies that may still be in flight time to land first.
-        if (*s_abort)
+        // After an abandoned wait: tell the other CTA of a pair to give up as well (its next poll
+        // sees the flag), then give copies and MMAs that may still be in flight time to finish.
+        if (*s_abort) {
+            if (kPair && threadIdx.x == kFirstEpiWarp * 32)
+                ptx::st_cluster_u32(ptx::map_to_cta(ptx::smem_u32(const_cast<int*>(s_abort)), rank ^ 1u), 1u);
             for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        }
         ptx::tc_fence_before();
         ptx::bar_sync(1, 4 * 32);
         if (warp == kFirstEpiWarp) {
@@ -546,14 +555,16 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             if (kPair) {
                 // Neither CTA may free TMEM, or leave, while the other still reads accumulators or
                 // sends signals here: tell the other CTA that this one is done, wait for its word.
+                // This wait ignores the abort flag: after an abort the other CTA still has to notice
+                // the flag, drain and send its word, which takes it at most one more wait limit.
                 if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(dealloc_bar, rank ^ 1u));
-                ptx::mbar_wait_warp<kPollNs>(dealloc_bar, 0, s_abort, kWaitLimitCycles);
+                ptx::mbar_wait_warp<kPollNs>(dealloc_bar, 0, s_never, 2 * max(P.wait_limit, kWaitLimitCycles));
                 ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
             } else {
                 ptx::tmem_dealloc(tmem_base, kTmemCols);
             }
         }
-        if (P.fold) {
+        if (P.fold == 1) {
             // ---------------------------------------------------------------- folded finalize
             // Whoever draws the last ticket knows that every CTA's partials are in global memory.
             const int tid_e = threadIdx.x - kFirstEpiWarp * 32;
@@ -782,6 +793,16 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
     return DM_OK;
 }
 
+int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
+                        void* out, uint32_t* err, cudaStream_t stream) {
+    if (head.dtype != DM_BF16 || head.d % 8 != 0) return DM_EUNSUPPORTED;
+    const long long n_threads = (long long)rows * (head.d / 8);
+    mask_operand_kernel<<<(unsigned)((n_threads + 255) / 256), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(H), static_cast<__nv_bfloat16*>(out), rows, head.d, map, mk.key0, mk.key1,
+        mk.thr, err);
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+}
+
 void fused_destroy(FusedState* fs) {
     if (fs == nullptr) return;
     cudaFree(fs->staging);
@@ -791,7 +812,8 @@ void fused_destroy(FusedState* fs) {
 int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hidden*/, int rows,
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
-                 const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out) {
+                 const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out,
+                 unsigned long long* packed_out, long long wait_limit) {
     if (folded_out) *folded_out = false;
     if (fs == nullptr || !fused_supported(head, rows) || fs->geo[0].n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
     // Slices of one-block launches: an even count (pairs need one); a CTA whose slice lies past the
@@ -863,9 +885,17 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.ticket = ticket;
         P.best = best;
         if (P.fold) { P.fin = *fin; if (folded_out) *folded_out = true; }
+        if (packed_out != nullptr && rows <= kMaxNPad) {
+            // one launch covers the call and the caller wants one packed word per path: reduce
+            // straight into the caller's array (which the caller has zeroed on this stream)
+            P.fold = 2;
+            P.best = packed_out;
+            if (folded_out) *folded_out = true;
+        }
         // Programmatic stream serialization, except when the row selection of the debug call could
         // itself be the output of the kernel ahead (it is read in the prologue).
         P.pdl = map.sel == nullptr ? 1 : 0;
+        P.wait_limit = wait_limit > 0 ? wait_limit : kWaitLimitCycles;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)grid);
         cfg.blockDim = dim3(kThreads);

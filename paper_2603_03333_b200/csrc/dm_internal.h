@@ -48,6 +48,9 @@ struct FinalizeArgs {
     int32_t* out_tokens;         // [B,T,K]
     int32_t* out_counts;         // [B,T,K]
     int32_t* out_accept_len;     // [B]
+    // device error word of the call's context (or null): if it is set when the results are about to
+    // be written, a kernel of the call gave up on a wait and the partial maxima mean nothing
+    const uint32_t* err;
 };
 
 // Reduce the per-slice partial argmaxes to one packed word per row (no histogram, no acceptance).
@@ -72,16 +75,22 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidd
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
-                 unsigned long long* best = nullptr, bool* folded_out = nullptr);
+                 unsigned long long* best = nullptr, bool* folded_out = nullptr,
+                 unsigned long long* packed_out = nullptr, long long wait_limit = 0);
+
+// The staged masked operand of the tensor-core kernel (Eq. 1 and the numerator of Eq. 2), written to `out`.
+int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
+                        void* out, uint32_t* err, cudaStream_t stream);
 
 int launch_read_stream(const void* ptr, size_t bytes, unsigned int* sink, int sms, cudaStream_t stream);
 
 // JS-divergence acceptance (Eq. 4, Eq. 5, Algorithm 1) on logits [B*T*K][V] written by a head kernel.
 int js_chunks(int V);
 size_t js_workspace_floats(int V, int max_rows, int max_hidden);
+constexpr int kJsMaxPositions = 65535;   // B*T of one JS call (a grid dimension)
 int launch_js(const float* logits, const float* draft_prob, float* workspace, int V, int B, int T, int K,
               const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
-              int32_t* out_accept_len, cudaStream_t stream);
+              int32_t* out_accept_len, const uint32_t* err, cudaStream_t stream);
 
 int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo, int shared_masks,
                        uint32_t* out_bits, cudaStream_t stream);

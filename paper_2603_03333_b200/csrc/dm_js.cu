@@ -246,9 +246,11 @@ js_sum_reg_kernel(const float* __restrict__ logits, const float* __restrict__ dr
 __global__ void __launch_bounds__(kJsThreads)
 js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, const int32_t* __restrict__ tokens,
                  const int32_t* __restrict__ draft, float* __restrict__ out_js, int32_t* __restrict__ out_js_ok,
-                 int32_t* __restrict__ out_accept_len) {
+                 int32_t* __restrict__ out_accept_len, const uint32_t* __restrict__ err) {
     extern __shared__ int32_t ok[];   // [T]
     const int b = blockIdx.x;
+    // a kernel of this call gave up on a wait: the logits are incomplete, nothing may be accepted
+    const bool failed = err != nullptr && *reinterpret_cast<const volatile uint32_t*>(err) != 0u;
     // divergences: one warp per (position, series), lanes over the chunks, summed in double
     for (int x = threadIdx.x >> 5; x < T * (K + 1); x += kJsThreads / 32) {
         const size_t idx = (size_t)b * T * (K + 1) + x;
@@ -266,8 +268,8 @@ js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, co
         for (int i = 1; i < K; ++i) max_heads = fmaxf(max_heads, js[i]);
         const bool eq5 = js[K] <= max_heads;                                   // Eq. 5
         const bool eq6 = position_ok(tokens + q * K, K, draft[q], DM_RULE_MAJORITY, nullptr);   // Eq. 6
-        if (out_js_ok) out_js_ok[q] = eq5;
-        ok[t] = eq5 || eq6;
+        if (out_js_ok) out_js_ok[q] = eq5 && !failed;
+        ok[t] = (eq5 || eq6) && !failed;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -291,8 +293,9 @@ size_t js_workspace_floats(int V, int max_rows, int max_hidden) {
 
 int launch_js(const float* logits, const float* draft_prob, float* workspace, int V, int B, int T, int K,
               const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
-              int32_t* out_accept_len, cudaStream_t stream) {
+              int32_t* out_accept_len, const uint32_t* err, cudaStream_t stream) {
     const int n_pos = B * T, n_chunks = js_chunks(V);
+    if (n_pos > kJsMaxPositions) return DM_EUNSUPPORTED;   // positions are the grid's second dimension
     const int chunk_len = (V + n_chunks - 1) / n_chunks;
     float2* part = reinterpret_cast<float2*>(workspace);
     float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
@@ -312,8 +315,9 @@ int launch_js(const float* logits, const float* draft_prob, float* workspace, in
         js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K,
                                                                                       chunk_len, n_chunks, part, share);
     }
+    if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
     js_accept_kernel<<<B, kJsThreads, T * sizeof(int32_t), stream>>>(share, n_chunks, T, K, tokens, draft, out_js,
-                                                                  out_js_ok, out_accept_len);
+                                                                  out_js_ok, out_accept_len, err);
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 

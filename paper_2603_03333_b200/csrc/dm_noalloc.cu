@@ -106,6 +106,7 @@ extern "C" int dropmatch_verify_batched_static(int device, const void* W, int V,
         fa.draft = draft; fa.out_hits = out_draft_hits;
         fa.N = 0;
         fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+        fa.err = err;
         st = launch_finalize(partials, n_slices, (int)rows, fa, s);
     } while (false);
     if (st == DM_ECUDA) cudaGetLastError();

@@ -1,8 +1,10 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times.
 
-The oracle needs V*d fp64 multiply-adds per path (half a second at the Llama-3-8B head), so it is
-run on a sample of paths: their decoded tokens (outside near-ties) and their full logit rows are
-compared one by one.  Everything that is integer work is checked in full from the GPU's own
+The oracle needs V*d fp64 multiply-adds per path (half a second at the Llama-3-8B head).  The
+benchmarked call (Llama-3-8B head, 40 paths) is compared with it in full.  The larger calls are
+compared on a sample of paths spread evenly over the call's rows, so that every kernel launch
+and both row blocks of a two-block launch are hit: decoded tokens (outside near-ties) and full
+logit rows, one by one.  Everything that is integer work is checked in full from the GPU's own
 tokens with the oracle's integer routines: multiplicities, hits, accepted lengths, tree walks;
 masks are compared bit for bit on sampled paths."""
 import numpy as np
@@ -12,7 +14,7 @@ import torch
 import oracle
 import paper_2603_03333_b200 as pk
 from paper_2603_03333_b200 import binding, workloads as wl
-from parity_util import NEAR_TIE, TOL_LOGIT_BF16, to_np
+from parity_util import NEAR_TIE, TOL_LOGIT_BF16, check_chain, to_np
 
 pytestmark = pytest.mark.gpu
 SEED = wl.MASK_SEED
@@ -20,9 +22,12 @@ DEV = "cuda:0"
 
 
 def _sample_paths(cfg, n, rng):
-    all_paths = [(b, t, i) for b in range(cfg.B) for t in range(cfg.T) for i in range(cfg.K)]
-    idx = rng.choice(len(all_paths), size=min(n, len(all_paths)), replace=False)
-    return [all_paths[j] for j in sorted(idx)]
+    """n paths (b, t, i), one from each of n equal stretches of the call's rows (row = (b*T+t)*K+i):
+    every launch of up to 256 (or 2 x 256) rows gets its share."""
+    rows = cfg.rows
+    n = min(n, rows)
+    picks = sorted({min(rows - 1, int((k + rng.random()) * rows / n)) for k in range(n)})
+    return [(r // (cfg.T * cfg.K), (r // cfg.K) % cfg.T, r % cfg.K) for r in picks]
 
 
 def _check_sampled_paths(ctx, cfg, work, got_tokens, paths, seq_base=0):
@@ -50,10 +55,31 @@ def _check_masks(ctx, cfg, paths, seq_base=0):
         assert np.array_equal((got[b, t, i, js // 32] >> (js % 32)) & 1, bits)
 
 
+def test_bench_workload_every_path():
+    """The call bench.py times (Llama-3-8B head, B=1, T=5, K=8: 40 paths, one launch) against the
+    oracle's whole call: all 40 tokens, counts, hits and the accepted length."""
+    cfg = wl.CONFIGS["llama8b"]
+    work = wl.make_workload(cfg, device=DEV)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
+        got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
+        assert ctx.device_error() == 0 and ctx.last_impl() == binding.IMPL_TCGEN05 and ctx.last_launches() == 1
+        draft = work.draft.cpu().numpy()
+        ref = oracle.verify_batched(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H), draft,
+                                    cfg.K, cfg.p, SEED)
+        n_diff = check_chain(got, ref, draft)
+        near = int((ref["gap"] < NEAR_TIE).sum())
+        print(f"llama8b: {n_diff} of {cfg.rows} tokens differ, all inside the {near} near-tie rows")
+        assert n_diff <= near
+    finally:
+        ctx.close()
+
+
 @pytest.mark.parametrize("name,overrides,n_paths", [
-    ("llama8b", {}, 8),                               # the bench workload: one accumulator group, in-kernel masks
-    ("qwen8b", dict(K=16), 5),                        # 112 rows: staged operand, three groups
-    ("qwen8b", dict(K=32, p=0.2), 4),                 # 224 rows: two accumulator slots, exposed epilogue
+    ("llama8b", dict(K=32, T=8), 16),                 # 256 rows: staged operand, CTA pairs
+    ("qwen8b", dict(K=16), 8),                        # 112 rows: staged operand, three groups
+    ("qwen8b", dict(K=32, p=0.2), 8),                 # 224 rows: two accumulator slots, exposed epilogue
 ])
 def test_chain_configs_at_full_size(name, overrides, n_paths):
     cfg = wl.CONFIGS[name].with_(**overrides)
@@ -96,7 +122,7 @@ def test_tree_config_at_full_size():
             assert 0 <= L <= 7
             for q in range(cfg.T):
                 assert np.array_equal(got["counts"][b, q], oracle.counts(got["tokens"][b, q], -1)[0])
-        paths = _sample_paths(cfg, 4, np.random.default_rng(12))
+        paths = _sample_paths(cfg, 32, np.random.default_rng(12))   # several paths in every launch and row block
         _check_sampled_paths(ctx, cfg, work, got["tokens"], paths)
     finally:
         ctx.close()
@@ -113,7 +139,7 @@ def test_llama70b_config_sampled():
         draft = work.draft.cpu().numpy()
         for b in range(cfg.B):
             assert got["accept_len"][b] == oracle.accept_chain(got["tokens"][b], draft[b], oracle.RULE_NAIVE)
-        paths = _sample_paths(cfg, 3, np.random.default_rng(13))
+        paths = _sample_paths(cfg, 32, np.random.default_rng(13))   # 2048 rows: four two-block launches, eight paths each
         _check_sampled_paths(ctx, cfg, work, got["tokens"], paths)
     finally:
         ctx.close()

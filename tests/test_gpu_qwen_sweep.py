@@ -3,8 +3,8 @@ B=1, and K=8, p=0.1 at B=8 and B=32, each at full size in the bench launch confi
 
 One head is built once for the module.  Per point: integer stages (counts, hits, accepted
 lengths) are checked in full from the GPU's own tokens with the oracle's integer routines, the
-tokens must lie in the vocabulary, and sampled paths are compared one by one with the oracle
-(token outside near-ties, full logit row within the bf16 bound)."""
+tokens must lie in the vocabulary, and eight paths spread evenly over the call's rows are compared
+one by one with the oracle (token outside near-ties, full logit row within the bf16 bound)."""
 import numpy as np
 import pytest
 import torch
@@ -45,7 +45,9 @@ def test_qwen_sweep_point(head, B, K, p):
             assert np.array_equal(got["counts"][b, t], cnt) and got["hits"][b, t] == hits
         assert got["accept_len"][b] == oracle.accept_chain(got["tokens"][b], draft[b], oracle.RULE_NAIVE)
     rng = np.random.default_rng(1000 * B + 10 * K + int(100 * p))
-    paths = sorted({(int(rng.integers(B)), int(rng.integers(cfg.T)), int(rng.integers(K))) for _ in range(2)})
+    # eight paths, one from each eighth of the call's rows (every launch and row block is hit)
+    rows = [min(cfg.rows - 1, int((k + rng.random()) * cfg.rows / 8)) for k in range(8)]
+    paths = sorted({(r // (cfg.T * K), (r // K) % cfg.T, r % K) for r in rows})
     Hn = wl.to_numpy_storage(work.H)
     sel = torch.tensor(paths, dtype=torch.int32, device=DEV)
     logits = ctx.debug_logits(work.H, sel, p, SEED, seq_base=11).cpu().numpy()

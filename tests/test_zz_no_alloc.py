@@ -2,14 +2,16 @@
 when they verify (a server whose pool owns all of HBM, a decode loop that may not stall on
 cudaMalloc, a plug-in without a context of its own).  It must give exactly what the context-based
 call gives on the same kernel family, call after call, although every call reuses one fixed
-scratch array inside the library.  Collected last on purpose: a stop-at-first-failure run has
-then already run every other test."""
+scratch array inside the library; and both are refereed by the CPU oracle.  Collected last on
+purpose: a stop-at-first-failure run has then already run every other test."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2603_03333_b200 as pk
 from paper_2603_03333_b200 import binding, workloads as wl
+from parity_util import check_chain
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -40,6 +42,10 @@ def test_static_entry_point_matches_context_entry_point_twice(cfg, rule):
             got = _np(out)
             for key in KEYS:   # integer results of the same kernels on the same inputs: bit-exact
                 assert np.array_equal(got[key], want[key]), (call, key)
+            draft = work.draft.cpu().numpy()
+            ref = oracle.verify_batched(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H), draft,
+                                        cfg.K, cfg.p, seed, seq_base=5, rule=rule)
+            check_chain(got, ref, draft, rule)   # and what the oracle computes from Eq. 1-3 and Sec. 3.2
         assert ctx.device_error() == 0
     finally:
         ctx.close()
