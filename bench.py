@@ -1,9 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the DropMatch verification path: verify calls/s on the Llama-3-8B-shaped head.
 
-One step = one whole verify call (masked head kernel + finalize kernel) on one batch of
-synthetic input: d=4096, V=128256, bf16, T=5 draft positions, K=8 dropout paths, p=0.1, B=1.
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+One step = one whole verify call (Eq. 1 masks, Eq. 2-3 masked head, per-path argmax, token
+counts, acceptance scan: one launch of the fused kernel at this size) on one batch of synthetic
+input: d=4096, V=128256, bf16, T=5 draft positions, K=8 dropout paths, p=0.1, B=1.
+Prints ONE JSON line (rank 0).  `--gpus N` run as plain `python bench.py` starts N ranks itself
+(one per GPU, independent replicas); under torchrun it joins the ranks it is given.
+`--impl reference` times the CPU oracle instead.
 """
 from __future__ import annotations
 
@@ -129,6 +132,42 @@ def aggregate_calls_per_s(ms_total_local: float, steps: int, world: int, device=
     return world * steps / (ms_total * 1e-3), ms_total / steps
 
 
+def parity_report(cfg, got_tokens, work_cpu):
+    """One full comparison of a call's decoded tokens with the CPU oracle, outside every timed
+    region: how many rows the oracle itself flags as near-ties (top-2 logit gap below 2e-2) and
+    how many tokens differ (allowed only inside those rows)."""
+    import oracle
+    from paper_2603_03333_b200 import workloads as wl
+    ref = oracle.verify_batched(wl.to_numpy_storage(work_cpu.W), cfg.dtype, wl.to_numpy_storage(work_cpu.H),
+                                work_cpu.draft.numpy(), cfg.K, cfg.p, wl.MASK_SEED)
+    differ = got_tokens != ref["tokens"]
+    near = ref["gap"] < 2e-2
+    return dict(rows_compared=int(differ.size), near_tie_rows=int(near.sum()), token_mismatches=int(differ.sum()),
+                mismatches_outside_near_ties=int((differ & ~near).sum()), near_tie_gap=2e-2)
+
+
+def self_launch(args) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script (one per GPU,
+    rendezvous on 127.0.0.1) and pass rank 0's JSON line through."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(args.gpus):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(args.gpus),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "INFO")           # the communicator log (stderr) shows the rank count
+        env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        procs.append(subprocess.Popen([sys.executable, str(Path(__file__).resolve()), *sys.argv[1:]], env=env,
+                                      stdout=subprocess.PIPE if rank == 0 else subprocess.DEVNULL, text=True))
+    out, _ = procs[0].communicate()
+    rcs = [procs[0].returncode] + [p.wait() for p in procs[1:]]
+    sys.stdout.write(out)
+    sys.stdout.flush()
+    return max(abs(rc) for rc in rcs)
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -157,12 +196,15 @@ def run_cuda(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    backend = os.environ.get("DM_BENCH_BACKEND", "nccl")   # "gloo" + DM_BENCH_STUB: launcher test on CPU
+    if os.environ.get("DM_BENCH_STUB"):
+        return run_stub(args, rank, world, backend)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the verification path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+        dist.init_process_group(backend, device_id=torch.device(dev))
 
     cfg = wl.CONFIGS[args.workload]
     work = wl.make_workload(cfg, device=dev)       # every rank: an independent replica of the call
@@ -276,6 +318,10 @@ def run_cuda(args):
         work_cpu = wl.Workload(cfg, work.W.cpu(), work.H.cpu(), work.draft.cpu(), None, None, None)
         v, cores, sample, _ = time_oracle(cfg, work_cpu, steps=1, warmup=0, budget_s=15.0)
         line["cpu_baseline"] = dict(value=v, unit=UNIT, cores=cores, kind="oracle", sample=sample)
+        if cfg.rows <= 64:     # the whole call through the oracle once more: seconds at this size
+            got = ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, wl.MASK_SEED, out=out)
+            torch.cuda.synchronize()
+            line["parity"] = parity_report(cfg, got["tokens"].cpu().numpy(), work_cpu)
     if rank == 0:
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -283,8 +329,22 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_stub(args, rank, world, backend):
+    """Launcher check without a GPU: every rank 'times' a fixed duration and the ranks aggregate
+    exactly as the real run does; rank 0 prints a line with the rank count."""
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group(backend)
+    value, ms_step = aggregate_calls_per_s(100.0 * (rank + 1), args.steps, world)
+    if rank == 0:
+        print(json.dumps(dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+                              ms_per_step=ms_step, stub=True)), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 SWEEPS = {
-    # (head name, V, d, [(B, T, K), ...]): the row counts of the tables in the design notes
+    # (head name, V, d, [(B, T, K), ...]): call sizes from 8 paths to the tensor-bound range
     "llama8b": (128256, 4096, [(1, 1, 8), (1, 2, 8), (1, 5, 8), (1, 8, 8), (1, 5, 16), (1, 8, 16), (1, 5, 32),
                                (1, 8, 32), (3, 5, 20), (4, 8, 16), (8, 8, 16)]),
     "qwen8b": (151936, 4096, [(B, 7, K) for B in (1, 8, 32) for K in (4, 8, 16, 32)]),
@@ -343,6 +403,11 @@ def main():
     ap.add_argument("--sweep", default=None, choices=sorted(SWEEPS), help="time a list of call sizes on one head")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep:
+        if args.impl == "reference":
+            os.environ.update(RANK="0", WORLD_SIZE=str(args.gpus))     # rank 0 alone runs the oracle
+        else:
+            raise SystemExit(self_launch(args))
     if args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

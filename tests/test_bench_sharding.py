@@ -50,6 +50,22 @@ def test_two_gloo_ranks_report_the_slowest_replica():
         assert o["slowest"] == 2.0
 
 
+def test_plain_python_invocation_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` with no launcher around it: the script spawns two ranks, they
+    aggregate over gloo (stub step, no GPU), and exactly one JSON line with n_gpus = 2 comes back."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    env.update(DM_BENCH_STUB="1", DM_BENCH_BACKEND="gloo")
+    r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--steps", "10", "--warmup", "3"],
+                       env=env, capture_output=True, text=True, timeout=180)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2
+    assert abs(line["ms_per_step"] - 20.0) < 1e-9          # the slow stub rank: 200 ms over 10 steps
+    assert abs(line["value"] - 2 * 10 / 0.2) < 1e-6
+
+
 def test_single_rank_needs_no_process_group():
     import bench
     value, ms_step = bench.aggregate_calls_per_s(50.0, steps=10, world=1)
