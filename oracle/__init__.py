@@ -88,6 +88,18 @@ def lib() -> ctypes.CDLL:
         L.oracle_verify_js.argtypes = [vp, ci, ci, ci, vp, i32p, ctypes.POINTER(ctypes.c_float), ci, ci, ci, cf,
                                        u64, u64, i32p, i32p, f64p, i32p, i32p]
         L.oracle_verify_js.restype = None
+        cd = ctypes.c_double
+        L.oracle_sample_uniform.argtypes = [u64, u64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32]
+        L.oracle_sample_uniform.restype = cd
+        L.oracle_gumbel.argtypes = [cd]
+        L.oracle_gumbel.restype = cd
+        L.oracle_nucleus.argtypes = [f64p, ci, cd, cd, ctypes.POINTER(ctypes.c_ubyte)]
+        L.oracle_nucleus.restype = ci
+        L.oracle_sample_row.argtypes = [f64p, ci, cd, cd, u64, u64, ctypes.c_uint32, ctypes.c_uint32, f64p]
+        L.oracle_sample_row.restype = ci
+        L.oracle_verify_batched_sampled.argtypes = [vp, ci, ci, ci, vp, i32p, ci, ci, ci, cf, u64, u64, ci, cd, cd,
+                                                    i32p, f64p, i32p, i32p, i32p]
+        L.oracle_verify_batched_sampled.restype = None
         _lib = L
     return _lib
 
@@ -327,3 +339,51 @@ def verify_batched_next(W, dtype, H, draft, K, p, seed, seq_base=0, rule=RULE_NA
                                      nxt.ctypes.data_as(i32p))
     return dict(tokens=tokens, gap=gap, counts=cnt, hits=hits, accept_len=alen, plain=plain, plain_gap=pgap,
                 next=nxt)
+
+
+def sample_uniform(seed: int, s: int, t: int, i: int, v: int) -> float:
+    """The uniform variate in (0,1) behind the Gumbel noise of vocabulary entry v."""
+    return float(lib().oracle_sample_uniform(seed, s, t, i, v))
+
+
+def gumbel(u: float) -> float:
+    return float(lib().oracle_gumbel(float(u)))
+
+
+def nucleus(logits, temperature: float, top_p: float) -> np.ndarray:
+    """bool[V]: the tokens nucleus sampling may draw from Softmax(logits / temperature)."""
+    l = np.ascontiguousarray(logits, dtype=np.float64)
+    out = np.zeros(l.shape[0], dtype=np.uint8)
+    lib().oracle_nucleus(_f64p(l), l.shape[0], float(temperature), float(top_p),
+                         out.ctypes.data_as(ctypes.POINTER(ctypes.c_ubyte)))
+    return out.astype(bool)
+
+
+def sample_row(logits, temperature, top_p, seed, s, t, i):
+    """-> (token, gap): one draw of the sampling decode rule from a row of logits."""
+    l = np.ascontiguousarray(logits, dtype=np.float64)
+    gap = ctypes.c_double()
+    tok = lib().oracle_sample_row(_f64p(l), l.shape[0], float(temperature), float(top_p), seed, s, t, i,
+                                  ctypes.byref(gap))
+    return int(tok), float(gap.value)
+
+
+def verify_batched_sampled(W, dtype, H, draft, K, p, seed, temperature=1.0, top_p=1.0, seq_base=0, rule=RULE_NAIVE):
+    """verify_batched with every path's token drawn by the sampling decode rule instead of the argmax."""
+    Ws, Hs = _store(W, dtype), _store(H, dtype)
+    V, d = Ws.shape
+    B, T, d2 = Hs.shape
+    assert d2 == d
+    dr, drp = _i32(draft)
+    assert dr.shape == (B, T)
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    tokens = np.zeros((B, T, K), dtype=np.int32)
+    gap = np.zeros((B, T, K), dtype=np.float64)
+    cnt = np.zeros((B, T, K), dtype=np.int32)
+    hits = np.zeros((B, T), dtype=np.int32)
+    alen = np.zeros((B,), dtype=np.int32)
+    lib().oracle_verify_batched_sampled(Ws.ctypes.data, dtype, V, d, Hs.ctypes.data, drp, B, T, K,
+                                        float(np.float32(p)), seed, seq_base, rule, float(temperature), float(top_p),
+                                        tokens.ctypes.data_as(i32p), _f64p(gap), cnt.ctypes.data_as(i32p),
+                                        hits.ctypes.data_as(i32p), alen.ctypes.data_as(i32p))
+    return dict(tokens=tokens, gap=gap, counts=cnt, hits=hits, accept_len=alen)

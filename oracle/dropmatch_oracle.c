@@ -34,6 +34,10 @@
  * a scipy restatement of Algorithm 1 with both outcomes, p=0 collapse onto the centroid.
  * Next-token call: library fp64 GEMV argmax and a brute-force scan.  Shared masks: equal hidden
  * rows decode alike path by path, position t equals a one-position call.
+ * Sampling decode: the uniform variates against the Python-integer Philox; the nucleus against a
+ * numpy sort-and-cut; sampled tokens against a numpy Gumbel-max; token frequencies over many
+ * paths against the renormalised nucleus probabilities (chi-square) on vocabularies of up to 8;
+ * temperature -> 0 and top_p -> 0 reduce to the argmax.
  * Parity unpinned: the paper's printed aggregates (tau, agreement ratios) need
  * the authors' models and datasets and cannot pin anything here.
  */
@@ -339,6 +343,128 @@ void oracle_verify_tree(const void *W, int dtype, int V, int d, const void *H,
             node_hrow + (size_t)b * N, N, K, rule, out_node_ok ? out_node_ok + (size_t)b * N : NULL,
             out_best_node + b);
     }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Sampling decode rule (Sec. 3.2: the per-path token is the top-1 token "or"  */
+/* a token selected by nucleus sampling; the paper gives no parameters)        */
+/* ------------------------------------------------------------------------- */
+
+/* Uniform variate of vocabulary entry v for (sequence s, position t, path i): Philox4x32-10 at
+ * counter (v / 4, i + 2^31, t, s mod 2^32), key = seed, word v mod 4.  Path indices stay below
+ * 2^31, so these counters never meet the mask counters of Eq. 1.  The top 23 bits k of the word
+ * give u = (k + 0.5) / 2^23, which lies strictly inside (0,1) and is exact in fp32 and fp64. */
+double oracle_sample_uniform(uint64_t seed, uint64_t s, uint32_t t, uint32_t i, uint32_t v)
+{
+    uint32_t ctr[4] = { v >> 2, i | 0x80000000u, t, (uint32_t)s };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t w[4];
+    oracle_philox4x32_10(ctr, key, w);
+    return ((double)(w[v & 3u] >> 9) + 0.5) / 8388608.0;
+}
+
+/* Standard Gumbel variate g = -log(-log(u)). */
+double oracle_gumbel(double u)
+{
+    return -log(-log(u));
+}
+
+struct prob_index { double p; int v; };
+static int by_prob_desc(const void *a, const void *b)
+{
+    const struct prob_index *x = (const struct prob_index *)a, *y = (const struct prob_index *)b;
+    if (x->p > y->p) return -1;
+    if (x->p < y->p) return 1;
+    return x->v - y->v;   /* equal probabilities: smaller token id first */
+}
+
+/* Nucleus of a logit row: p = Softmax(l / temperature); tokens in order of decreasing p (equal p:
+ * increasing id) are taken until their cumulative probability reaches top_p, the token that
+ * crosses it included; top_p >= 1 keeps every token.  in_nucleus[v] = 1/0.  Returns the size. */
+int oracle_nucleus(const double *logits, int V, double temperature, double top_p, unsigned char *in_nucleus)
+{
+    if (top_p >= 1.0) {
+        memset(in_nucleus, 1, (size_t)V);
+        return V;
+    }
+    struct prob_index *ord = (struct prob_index *)malloc((size_t)V * sizeof *ord);
+    double zmax = -INFINITY, sum = 0.0;
+    for (int v = 0; v < V; ++v)
+        if (logits[v] / temperature > zmax) zmax = logits[v] / temperature;
+    for (int v = 0; v < V; ++v) {
+        ord[v].p = exp(logits[v] / temperature - zmax);
+        ord[v].v = v;
+        sum += ord[v].p;
+    }
+    for (int v = 0; v < V; ++v) ord[v].p /= sum;
+    qsort(ord, (size_t)V, sizeof *ord, by_prob_desc);
+    memset(in_nucleus, 0, (size_t)V);
+    double cum = 0.0;
+    int n = 0;
+    while (n < V) {
+        in_nucleus[ord[n].v] = 1;
+        cum += ord[n].p;
+        ++n;
+        if (cum >= top_p) break;
+    }
+    free(ord);
+    return n;
+}
+
+/* One sampled token: y = argmax over the nucleus of l[v] / temperature + g[v] (the Gumbel-max
+ * form of drawing from the renormalised nucleus distribution); equal keys go to the smaller id.
+ * gap = winning key - runner-up key within the nucleus (infinite if the nucleus is one token). */
+int oracle_sample_row(const double *logits, int V, double temperature, double top_p, uint64_t seed,
+                      uint64_t s, uint32_t t, uint32_t i, double *gap)
+{
+    unsigned char *in = (unsigned char *)malloc((size_t)V);
+    oracle_nucleus(logits, V, temperature, top_p, in);
+    int best = -1;
+    double best_key = -INFINITY, second = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        if (!in[v]) continue;
+        double key = logits[v] / temperature + oracle_gumbel(oracle_sample_uniform(seed, s, t, i, (uint32_t)v));
+        if (best < 0 || key > best_key) {
+            if (best >= 0) second = best_key;
+            best_key = key;
+            best = v;
+        } else if (key > second) {
+            second = key;
+        }
+    }
+    if (gap) *gap = best_key - second;
+    free(in);
+    return best;
+}
+
+/* Chain verification with the sampling decode rule in place of the argmax of Sec. 3.2: Eq. 1-3 as
+ * before, y^(i) drawn as above, then counts, per-position test and left-to-right scan unchanged.
+ * H[B,T,d], draft[B,T] -> tokens[B,T,K], gap[B,T,K] (may be NULL), counts, hits[B,T], accept_len[B]. */
+void oracle_verify_batched_sampled(const void *W, int dtype, int V, int d, const void *H,
+                                   const int32_t *draft, int B, int T, int K, float p, uint64_t seed,
+                                   uint64_t seq_base, int rule, double temperature, double top_p,
+                                   int32_t *out_tokens, double *out_gap, int32_t *out_counts,
+                                   int32_t *out_hits, int32_t *out_accept_len)
+{
+    const size_t elem = dtype == ORACLE_F32 ? 4 : 2;
+    double *logits = (double *)malloc((size_t)V * sizeof(double));
+    for (int b = 0; b < B; ++b) {
+        for (int t = 0; t < T; ++t) {
+            size_t q = (size_t)b * T + t;
+            const void *h_row = (const char *)H + q * d * elem;
+            for (int i = 0; i < K; ++i) {
+                double gap;
+                oracle_logits_row(W, dtype, V, d, h_row, p, seed, seq_base + (uint64_t)b, t, i, logits);
+                out_tokens[q * K + i] = oracle_sample_row(logits, V, temperature, top_p, seed,
+                                                          seq_base + (uint64_t)b, (uint32_t)t, (uint32_t)i, &gap);
+                if (out_gap) out_gap[q * K + i] = gap;
+            }
+            int hits = oracle_counts(out_tokens + q * K, K, draft[q], out_counts + q * K);
+            if (out_hits) out_hits[q] = hits;
+        }
+        out_accept_len[b] = oracle_accept_chain(out_tokens + (size_t)b * T * K, draft + (size_t)b * T, T, K, rule);
+    }
+    free(logits);
 }
 
 /* ------------------------------------------------------------------------- */
