@@ -116,6 +116,23 @@ int dropmatch_verify_batched(dm_ctx* ctx, const void* H, const int32_t* draft, i
                              int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
                              int32_t* out_accept_len, void* stream);
 
+/* dropmatch_verify_batched with the sampling decode rule: Sec. 3.2 lets the per-path token be the
+ * top-1 token "or" one selected by nucleus sampling, without giving parameters.  Here path i of
+ * position t draws y from Softmax(l / temperature) by the Gumbel-max construction,
+ *   y = argmax_v ( l[v] / temperature - log(-log(u[v])) ),   equal keys -> smaller id,
+ * with u[v] = (n + 0.5) / 2^23, n = top 23 bits of word (v mod 4) of
+ * Philox4x32-10(counter = (v/4, i + 2^31, t, s mod 2^32), key = seed): the same generator as the
+ * masks, on counters the masks never use, so a call is reproducible from (seed, s, t, i) alone.
+ * The noise is generated in the epilogue of the head kernel (one Philox call and two logarithms
+ * per logit); no logit is written to memory.  Counts, per-position test and scan are unchanged.
+ *   temperature > 0;  top_p in (0,1]: the nucleus mass.  top_p < 1 needs all logits of a path at
+ *   once (sort and cut) and is not implemented on the device: DM_EUNSUPPORTED.
+ * Everything else as for dropmatch_verify_batched. */
+int dropmatch_verify_batched_sampled(dm_ctx* ctx, const void* H, const int32_t* draft, int B, int T, int K,
+                                     float p, uint64_t seed, uint64_t seq_base, int rule, float temperature,
+                                     float top_p, int32_t* out_tokens, int32_t* out_counts,
+                                     int32_t* out_draft_hits, int32_t* out_accept_len, void* stream);
+
 /* dropmatch_verify_batched plus the token the engine emits after the accepted prefix.  Every
  * hidden row gets, in the same pass over W, one more path without dropout: the target model's own
  * greedy token (the paper does not say how DropMatch picks the correction or bonus token; this

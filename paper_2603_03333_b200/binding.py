@@ -35,6 +35,8 @@ SIGNATURES = {
     "dropmatch_finalize_packed": (_ci, [_vp, _vp, _ci, _vp, _ci, _ci, _ci, _ci, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _u64, _ci, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
+    "dropmatch_verify_batched_sampled": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _cf, _cf,
+                                               _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_next": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _ci, _cf, _u64, _u64, _ci,
                                             _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "dropmatch_verify_batched_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _ci, _vp, _vp, _vp, _vp, _vp]),
@@ -214,6 +216,19 @@ class Context:
                                               _ptr(out["tokens"]), _ptr(out["counts"]), _ptr(out["hits"]),
                                               _ptr(out["accept_len"]), _stream(self.device)),
                "dropmatch_verify_batched")
+        return out
+
+    # -- dropmatch_verify_batched_sampled
+    def verify_batched_sampled(self, H, draft, K, p, seed, temperature=1.0, top_p=1.0, seq_base=0, rule=RULE_NAIVE,
+                               out=None):
+        B, T, _ = H.shape
+        _dev(H, self._tdtype(), "H"); _dev(draft, torch.int32, "draft")
+        if out is None:
+            out = self.alloc_outputs(B, T, K)
+        _check(lib().dropmatch_verify_batched_sampled(self._h, _ptr(H), _ptr(draft), B, T, K, p, seed, seq_base, rule,
+                                                      temperature, top_p, _ptr(out["tokens"]), _ptr(out["counts"]),
+                                                      _ptr(out["hits"]), _ptr(out["accept_len"]),
+                                                      _stream(self.device)), "dropmatch_verify_batched_sampled")
         return out
 
     # -- dropmatch_verify_batched_next

@@ -76,6 +76,8 @@ bool make_mask_key(float p, uint64_t seed, MaskKey* mk) {
     mk->key0 = (uint32_t)seed;
     mk->key1 = (uint32_t)(seed >> 32);
     mk->scale = (float)(1.0 / (1.0 - (double)p));
+    mk->sample = 0;
+    mk->inv_temp = 1.0f;
     return true;
 }
 
@@ -335,6 +337,32 @@ int dropmatch_verify_batched(dm_ctx* c, const void* H, const int32_t* draft, int
     if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
     MaskKey mk;
     if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return DM_ECUDA;
+    RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};
+    FinalizeArgs fa{};
+    fa.B = B; fa.T = T; fa.K = K; fa.rule = rule;
+    fa.draft = draft; fa.out_hits = out_draft_hits;
+    fa.N = 0;
+    fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
+    return run_verify(c, H, B * T * K, map, mk, fa, static_cast<cudaStream_t>(stream));
+}
+
+int dropmatch_verify_batched_sampled(dm_ctx* c, const void* H, const int32_t* draft, int B, int T, int K, float p,
+                                     uint64_t seed, uint64_t seq_base, int rule, float temperature, float top_p,
+                                     int32_t* out_tokens, int32_t* out_counts, int32_t* out_draft_hits,
+                                     int32_t* out_accept_len, void* stream) {
+    int st = check_common(c, H, B, T, K);
+    if (st != DM_OK) return st;
+    if (draft == nullptr || out_tokens == nullptr || out_counts == nullptr || out_accept_len == nullptr)
+        return DM_EINVAL;
+    if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
+    if (!(temperature > 0.0f) || !(temperature < 1e30f) || !(top_p > 0.0f) || !(top_p <= 1.0f)) return DM_EINVAL;
+    if (top_p < 1.0f) return DM_EUNSUPPORTED;   // the nucleus cut needs every logit of a path at once
+    MaskKey mk;
+    if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
+    mk.sample = 1;
+    mk.inv_temp = 1.0f / temperature;
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
     RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};

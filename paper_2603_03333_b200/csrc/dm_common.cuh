@@ -86,6 +86,19 @@ __device__ __forceinline__ uint32_t keep4(uint32_t quad, const RowKey& k, uint32
            (w.w >= thr ? 8u : 0u);
 }
 
+// Sampling decode rule (Sec. 3.2 names nucleus sampling as the alternative to the top-1 token):
+// Gumbel noise of vocabulary entry v for the path with key k.  Philox counter (v / 4, i + 2^31,
+// t, s), word v mod 4: path indices stay below 2^31, so these counters never meet the mask
+// counters.  The top 23 bits n of the word give u = (n + 0.5) / 2^23, exact in fp32 and strictly
+// inside (0,1); g = -log(-log(u)) is a standard Gumbel variate, and the argmax of
+// logit / temperature + g is a draw from Softmax(logits / temperature).
+__device__ __forceinline__ float gumbel_noise(uint32_t v, const RowKey& k, uint32_t key0, uint32_t key1) {
+    const uint4 w = philox4x32_10(make_uint4(v >> 2, k.i | 0x80000000u, k.t, k.s), key0, key1);
+    const uint32_t word = (v & 2u) ? ((v & 1u) ? w.w : w.z) : ((v & 1u) ? w.y : w.x);
+    const float u = ((float)(word >> 9) + 0.5f) * 1.1920928955078125e-07f;   // 2^-23
+    return -logf(-logf(u));
+}
+
 // Monotone map float -> uint32 (larger float <=> larger key); -0 is folded into +0 first so
 // that equal logits get equal keys.  NaN inputs are not expected (finite W and H).
 __device__ __forceinline__ uint32_t float_key(float x) {

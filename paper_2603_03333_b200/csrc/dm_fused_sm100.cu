@@ -79,6 +79,8 @@ struct FusedParams {
     RowMap map;
     uint32_t key0, key1, thr;
     float scale;
+    int sample;       // the epilogue adds Gumbel noise to logit * inv_temp before the maximum (sampling decode)
+    float inv_temp;
     unsigned long long* partials;   // [vocabulary slice][rows_total]
     float* dbg_logits;              // [rows_total][V] or null
     uint32_t* err;
@@ -452,10 +454,26 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                     ptx::tmem_ld16(tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)(slot * P.n_pad + n0), acc);
                     ptx::tmem_ld_wait();
                     if (++slot == P.n_slots) slot = 0;
+                    if (P.sample) {
+                        // sampling decode: one Philox call and two logarithms per logit
+                        if (valid) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float val = __uint_as_float(acc[j]) * P.scale;
-                        if (valid && val > best[j]) { best[j] = val; bv[j] = v; }
+                            for (int j = 0; j < 16; ++j) {
+                                if (n0 + j < my_rows) {
+                                    const RowInfo ri = s_row[n0 + j];
+                                    const RowKey k{0, ri.s, ri.t, ri.i};
+                                    const float val = fmaf(__uint_as_float(acc[j]) * P.scale, P.inv_temp,
+                                                           gumbel_noise((uint32_t)(v + P.v_offset), k, P.key0, P.key1));
+                                    if (val > best[j]) { best[j] = val; bv[j] = v; }
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float val = __uint_as_float(acc[j]) * P.scale;
+                            if (valid && val > best[j]) { best[j] = val; bv[j] = v; }
+                        }
                     }
                     if (P.dbg_logits != nullptr && valid) {
 #pragma unroll
@@ -878,6 +896,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.off_rowinfo = plan.off_rowinfo; P.off_best = plan.off_best; P.off_bar = plan.off_bar;
         P.map = map;
         P.key0 = mk.key0; P.key1 = mk.key1; P.thr = mk.thr; P.scale = mk.scale;
+        P.sample = mk.sample; P.inv_temp = mk.inv_temp;
         P.partials = partials; P.dbg_logits = dbg_logits; P.err = err;
         // a call of one launch finishes itself; larger calls leave it to finalize_kernel
         P.fold = (fin != nullptr && ticket != nullptr && best != nullptr && rows <= kMaxNPad &&

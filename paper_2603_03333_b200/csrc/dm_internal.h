@@ -25,6 +25,8 @@ struct MaskKey {
     uint32_t key0, key1;  // Philox key = seed
     uint32_t thr;         // drop iff word < thr; thr = floor(p * 2^32)
     float scale;          // 1 / (1 - p)
+    int sample;           // 0: argmax decode; 1: draw from Softmax(logits / temperature) by Gumbel-max
+    float inv_temp;       // 1 / temperature (sample == 1)
 };
 
 // Acceptance inputs/outputs handed to the finalize kernel.

@@ -93,6 +93,8 @@ extern "C" int dropmatch_verify_batched_static(int device, const void* W, int V,
         mk.key0 = (uint32_t)seed;
         mk.key1 = (uint32_t)(seed >> 32);
         mk.scale = (float)(1.0 / (1.0 - (double)p));
+        mk.sample = 0;
+        mk.inv_temp = 1.0f;
 
         static_scratch_reset_kernel<<<1, 1, 0, s>>>();
         if (cudaGetLastError() != cudaSuccess) { st = DM_ECUDA; break; }

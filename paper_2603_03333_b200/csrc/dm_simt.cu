@@ -34,7 +34,7 @@ template <> struct Vec<__nv_bfloat16> {
 template <typename T, int RC>
 __global__ void __launch_bounds__(256)
 simt_head_kernel(const T* __restrict__ W, const T* __restrict__ H, int V, int d, int rows,
-                 RowMap map, uint32_t key0, uint32_t key1, uint32_t thr, float scale,
+                 RowMap map, uint32_t key0, uint32_t key1, uint32_t thr, float scale, int sample, float inv_temp,
                  int v_per_block, int v_offset, unsigned long long* __restrict__ partials,
                  float* __restrict__ dbg_logits, uint32_t* __restrict__ err) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -97,6 +97,11 @@ simt_head_kernel(const T* __restrict__ W, const T* __restrict__ H, int V, int d,
                         dbg_logits[(size_t)(r0 + rr) * V + v] =
                             row_valid[rr] ? s : __uint_as_float(0x7FC00000u);
                     if (lane == rr) {
+                        if (sample) {   // sampling decode: Gumbel-max on logit / temperature
+                            RowKey k;
+                            row_key(map, r0 + rr, k);
+                            s = fmaf(s, inv_temp, gumbel_noise((uint32_t)(v + v_offset), k, key0, key1));
+                        }
                         unsigned long long cand = pack_best(float_key(s), (uint32_t)(v + v_offset));
                         best = cand > best ? cand : best;
                     }
@@ -128,7 +133,7 @@ static int launch_simt_rc(const HeadDesc& head, const void* H, int rows, const R
         return DM_ECUDA;
     kern<<<n_slices, 256, smem, stream>>>(static_cast<const T*>(head.W), static_cast<const T*>(H),
                                           head.V, head.d, rows, map, mk.key0, mk.key1, mk.thr,
-                                          mk.scale, v_per_block, head.v_offset, partials, dbg_logits, err);
+                                          mk.scale, mk.sample, mk.inv_temp, v_per_block, head.v_offset, partials, dbg_logits, err);
     if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
     *n_slices_out = n_slices;
     return DM_OK;
