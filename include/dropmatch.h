@@ -152,10 +152,14 @@ int dropmatch_verify_batched_next(dm_ctx* ctx, const void* H, const int32_t* dra
                                   void* stream);
 
 /* Same as dropmatch_verify_batched, but H, draft and all outputs are HOST pointers (pinned or
- * pageable).  Gathers the inputs in the context's pinned buffer and sends them with one copy,
- * runs the call with its outputs going to pinned memory the device can write, waits for
- * `stream`, and copies the results to the caller's arrays.  Needs B*T <= max_hidden_rows of
- * dm_set_head.  out_draft_hits may be NULL. */
+ * pageable).  Pinned buffers (cudaHostAlloc, cudaHostRegister, torch pin_memory) are used where
+ * they are: a small kernel fetches the inputs over the host link while the head kernel already
+ * streams W, and the results are written by the device straight into the caller's arrays.
+ * Pageable buffers go through the context's own pinned buffers (one memcpy each way).  The call
+ * returns after `stream` has drained, with the results in place.  Whether a pointer is pinned is
+ * looked up once and remembered (the last eight pointers): do not unpin or free a buffer and
+ * reuse its address as pageable memory without a dm_set_head in between.  Needs
+ * B*T <= max_hidden_rows of dm_set_head; H_host 16-byte aligned.  out_draft_hits may be NULL. */
 int dropmatch_verify_batched_host(dm_ctx* ctx, const void* H_host, const int32_t* draft_host, int B,
                                   int T, int K, float p, uint64_t seed, uint64_t seq_base, int rule,
                                   int32_t* out_tokens_host, int32_t* out_counts_host,

@@ -24,10 +24,15 @@ struct dm_ctx {
     // the same layout, H then the draft tokens; and a pinned, device-mapped buffer that the
     // kernels write the results into (tokens | counts | hits | accept_len)
     unsigned char* stage_in = nullptr;       // device
-    unsigned char* pin_in = nullptr;         // pinned host
+    unsigned char* pin_in = nullptr;         // pinned host, mapped
+    unsigned char* pin_in_dev = nullptr;     // the same memory as the device sees it
     int32_t* pin_out = nullptr;              // pinned host, mapped
     int32_t* pin_out_dev = nullptr;          // the same memory as the device sees it
     size_t ws_bytes = 0;
+    // host pointers the host-buffer entry point has already looked up: device alias, or null if pageable
+    struct HostAlias { const void* host = nullptr; void* dev = nullptr; };
+    HostAlias aliases[8];
+    int alias_next = 0;
     FusedState* fused = nullptr;             // tensor maps etc. of the tcgen05 kernel
     // JS criterion (dm_enable_js): logits of every path of a call, and the kernels' partial sums
     float* js_logits = nullptr;              // [js_max_rows][V]
@@ -59,6 +64,7 @@ void free_workspace(dm_ctx* c) {
     cudaFree(c->partials); c->partials = nullptr;
     cudaFree(c->stage_in); c->stage_in = nullptr;
     cudaFreeHost(c->pin_in); c->pin_in = nullptr;
+    c->pin_in_dev = nullptr;
     cudaFreeHost(c->pin_out); c->pin_out = nullptr;
     c->pin_out_dev = nullptr;
     if (c->fused) { fused_destroy(c->fused); c->fused = nullptr; }
@@ -66,6 +72,21 @@ void free_workspace(dm_ctx* c) {
     cudaFree(c->js_ws); c->js_ws = nullptr;
     c->js_max_rows = c->js_max_hidden = 0;
     c->ws_bytes = 0;
+}
+
+// Device-side alias of a host pointer if the memory is pinned (page-locked and readable and writable by the
+// device), else null.  Looked up once per pointer and remembered: the lookup costs about a microsecond.
+void* device_alias(dm_ctx* c, const void* host) {
+    for (const dm_ctx::HostAlias& a : c->aliases)
+        if (a.host == host) return a.dev;
+    cudaPointerAttributes attr{};
+    void* dev = nullptr;
+    if (cudaPointerGetAttributes(&attr, host) == cudaSuccess && attr.type == cudaMemoryTypeHost)
+        dev = attr.devicePointer;
+    cudaGetLastError();
+    c->aliases[c->alias_next] = dm_ctx::HostAlias{host, dev};
+    c->alias_next = (c->alias_next + 1) % 8;
+    return dev;
 }
 
 bool make_mask_key(float p, uint64_t seed, MaskKey* mk) {
@@ -213,10 +234,12 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
     const size_t n_in = (size_t)max_hidden_rows * d * elem + 16 + (size_t)max_hidden_rows * sizeof(int32_t);
     const size_t n_out = ((size_t)2 * max_hidden_rows + 2 * (size_t)max_rows) * sizeof(int32_t);
     void* out_dev = nullptr;
+    void* in_dev = nullptr;
     if (cudaMalloc(&c->partials, n_part) != cudaSuccess || cudaMalloc(&c->stage_in, n_in) != cudaSuccess ||
-        cudaHostAlloc(reinterpret_cast<void**>(&c->pin_in), n_in, cudaHostAllocDefault) != cudaSuccess ||
+        cudaHostAlloc(reinterpret_cast<void**>(&c->pin_in), n_in, cudaHostAllocMapped) != cudaSuccess ||
         cudaHostAlloc(reinterpret_cast<void**>(&c->pin_out), n_out, cudaHostAllocMapped) != cudaSuccess ||
         cudaHostGetDevicePointer(&out_dev, c->pin_out, 0) != cudaSuccess ||
+        cudaHostGetDevicePointer(&in_dev, c->pin_in, 0) != cudaSuccess ||
         cudaMemset(c->partials + (size_t)kMaxSlices * max_rows, 0, (size_t)max_rows * sizeof(unsigned long long)) !=
             cudaSuccess) {
         cudaGetLastError();
@@ -224,6 +247,8 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
         return DM_ECUDA;
     }
     c->pin_out_dev = static_cast<int32_t*>(out_dev);
+    c->pin_in_dev = static_cast<unsigned char*>(in_dev);
+    for (dm_ctx::HostAlias& a : c->aliases) a = dm_ctx::HostAlias{};
     c->ws_bytes = n_part + n_in;
     c->head = HeadDesc{W, V, d, dtype, 0};
     c->max_rows = max_rows;
@@ -427,32 +452,41 @@ int dropmatch_verify_batched_host(dm_ctx* c, const void* H_host, const int32_t* 
     if (!g.ok) return DM_ECUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t elem = c->head.dtype == DM_F32 ? 4 : 2;
-    // inputs: gathered in pinned memory, one host-to-device copy
     const size_t h_bytes = (size_t)hidden * c->head.d * elem;
     const size_t draft_off = (h_bytes + 15) & ~static_cast<size_t>(15);
-    memcpy(c->pin_in, H_host, h_bytes);
-    memcpy(c->pin_in + draft_off, draft_host, (size_t)hidden * sizeof(int32_t));
-    if (cudaMemcpyAsync(c->stage_in, c->pin_in, draft_off + (size_t)hidden * sizeof(int32_t), cudaMemcpyHostToDevice, s) !=
-        cudaSuccess) {
-        cudaGetLastError();
-        return DM_ECUDA;
+    // Inputs.  Pinned caller buffers are read by the device where they are; pageable ones are
+    // first gathered in the context's pinned buffer.  A small kernel then brings them over the
+    // host link into the device staging buffer while the head kernel already streams W.
+    const void* h_src = device_alias(c, H_host);
+    const void* d_src = device_alias(c, draft_host);
+    if (h_src == nullptr) {
+        memcpy(c->pin_in, H_host, h_bytes);
+        h_src = c->pin_in_dev;
     }
-    // outputs: the kernels write them straight into mapped pinned memory (a few hundred bytes
-    // crossing to the host), so no device-to-host copy has to be queued behind the kernel
-    int32_t* o_tok = c->pin_out;
-    int32_t* o_cnt = o_tok + rows;
-    int32_t* o_hits = o_cnt + rows;
-    int32_t* o_len = o_hits + hidden;
+    if (d_src == nullptr) {
+        memcpy(c->pin_in + draft_off, draft_host, (size_t)hidden * sizeof(int32_t));
+        d_src = c->pin_in_dev + draft_off;
+    }
+    int32_t* draft_dev = reinterpret_cast<int32_t*>(c->stage_in + draft_off);
+    st = launch_host_gather(h_src, h_bytes, static_cast<const int32_t*>(d_src), (int)hidden, c->stage_in, draft_dev, s);
+    if (st != DM_OK) return st;
+    // Outputs.  The kernels write them into host memory the device can reach (a few hundred bytes
+    // crossing to the host), so that no device-to-host copy is queued behind the call: straight into
+    // the caller's arrays if those are pinned, else into the context's mapped buffer.
+    int32_t* o_tok = static_cast<int32_t*>(device_alias(c, out_tokens_host));
+    int32_t* o_cnt = static_cast<int32_t*>(device_alias(c, out_counts_host));
+    int32_t* o_len = static_cast<int32_t*>(device_alias(c, out_accept_len_host));
+    int32_t* o_hits = out_draft_hits_host ? static_cast<int32_t*>(device_alias(c, out_draft_hits_host)) : nullptr;
     int32_t* d_out = c->pin_out_dev;
-    st = dropmatch_verify_batched(c, c->stage_in, reinterpret_cast<const int32_t*>(c->stage_in + draft_off), B, T, K, p,
-                                  seed, seq_base, rule, d_out, d_out + rows, d_out + 2 * rows, d_out + 2 * rows + hidden,
-                                  stream);
+    st = dropmatch_verify_batched(c, c->stage_in, draft_dev, B, T, K, p, seed, seq_base, rule,
+                                  o_tok ? o_tok : d_out, o_cnt ? o_cnt : d_out + rows,
+                                  o_hits ? o_hits : d_out + 2 * rows, o_len ? o_len : d_out + 2 * rows + hidden, stream);
     if (st != DM_OK) return st;
     if (cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
-    memcpy(out_tokens_host, o_tok, (size_t)rows * sizeof(int32_t));
-    memcpy(out_counts_host, o_cnt, (size_t)rows * sizeof(int32_t));
-    memcpy(out_accept_len_host, o_len, (size_t)B * sizeof(int32_t));
-    if (out_draft_hits_host) memcpy(out_draft_hits_host, o_hits, (size_t)hidden * sizeof(int32_t));
+    if (!o_tok) memcpy(out_tokens_host, c->pin_out, (size_t)rows * sizeof(int32_t));
+    if (!o_cnt) memcpy(out_counts_host, c->pin_out + rows, (size_t)rows * sizeof(int32_t));
+    if (!o_len) memcpy(out_accept_len_host, c->pin_out + 2 * rows + hidden, (size_t)B * sizeof(int32_t));
+    if (out_draft_hits_host && !o_hits) memcpy(out_draft_hits_host, c->pin_out + 2 * rows, (size_t)hidden * sizeof(int32_t));
     return DM_OK;
 }
 

@@ -60,6 +60,31 @@ int launch_finalize(const unsigned long long* partials, int n_slices, int rows,
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 
+// Host-buffer entry point: fetch a call's inputs (a few tens of KB) from pinned host memory that
+// the device can read and put them where the head kernel expects them.  The head kernel behind
+// this one may be scheduled at once: it streams W until its builders need H, and they wait for
+// this kernel to finish, so the trip over the host link hides behind the fill of the W ring.
+__global__ void __launch_bounds__(256)
+host_gather_kernel(const uint4* __restrict__ src_h, size_t n16, const int32_t* __restrict__ src_draft, int n_draft,
+                   uint4* __restrict__ dst_h, int32_t* __restrict__ dst_draft) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x; x < n16; x += stride) dst_h[x] = src_h[x];
+    for (size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x; x < (size_t)n_draft; x += stride)
+        dst_draft[x] = src_draft[x];
+}
+
+int launch_host_gather(const void* src_h, size_t h_bytes, const int32_t* src_draft, int n_draft, void* dst_h,
+                       int32_t* dst_draft, cudaStream_t stream) {
+    const size_t n16 = h_bytes / 16;
+    size_t blocks = (n16 + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 592) blocks = 592;
+    host_gather_kernel<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const uint4*>(src_h), n16, src_draft, n_draft,
+                                                           static_cast<uint4*>(dst_h), dst_draft);
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+}
+
 // Measurement aid: a plain read-only stream over a buffer (16-byte loads, grid-stride, XOR-folded
 // so that the loads cannot be dropped).  Its rate is the read-only HBM ceiling of the part.
 __global__ void __launch_bounds__(1024, 2)

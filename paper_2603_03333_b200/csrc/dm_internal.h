@@ -84,6 +84,10 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidd
 int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
                         void* out, uint32_t* err, cudaStream_t stream);
 
+// Copy a call's inputs from device-readable host memory into the device staging buffer (a kernel, not a DMA copy).
+int launch_host_gather(const void* src_h, size_t h_bytes, const int32_t* src_draft, int n_draft, void* dst_h,
+                       int32_t* dst_draft, cudaStream_t stream);
+
 int launch_read_stream(const void* ptr, size_t bytes, unsigned int* sink, int sms, cudaStream_t stream);
 
 // JS-divergence acceptance (Eq. 4, Eq. 5, Algorithm 1) on logits [B*T*K][V] written by a head kernel.

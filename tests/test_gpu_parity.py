@@ -186,10 +186,20 @@ def test_host_entry_point_equals_device_entry_point(ctx):
     ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
     dev = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=1))
     Hh, dh = work.H.cpu().pin_memory(), work.draft.cpu().pin_memory()
-    for _ in range(2):
+    for _ in range(2):        # pinned inputs and outputs: the device reads and writes them in place
         host = ctx.verify_batched_host(Hh, dh, cfg.K, cfg.p, SEED, seq_base=1)
         for key in ("tokens", "counts", "hits", "accept_len"):
             assert np.array_equal(host[key].numpy(), dev[key]), key
+    Hp, dp = work.H.cpu().clone(), work.draft.cpu().clone()      # pageable inputs and outputs: staged by the library
+    for _ in range(2):
+        out = ctx.alloc_host_outputs(cfg.B, cfg.T, cfg.K, pin=False)
+        host = ctx.verify_batched_host(Hp, dp, cfg.K, cfg.p, SEED, seq_base=1, out=out)
+        for key in ("tokens", "counts", "hits", "accept_len"):
+            assert np.array_equal(host[key].numpy(), dev[key]), key
+    mixed = ctx.alloc_host_outputs(cfg.B, cfg.T, cfg.K, pin=False)   # pinned inputs, pageable outputs
+    host = ctx.verify_batched_host(Hh, dh, cfg.K, cfg.p, SEED, seq_base=1, out=mixed)
+    for key in ("tokens", "counts", "hits", "accept_len"):
+        assert np.array_equal(host[key].numpy(), dev[key]), key
     with pytest.raises(pk.DropMatchError) as e:
         big = torch.zeros((cfg.B + 1, cfg.T, cfg.d), dtype=torch.bfloat16)
         ctx.verify_batched_host(big, torch.zeros((cfg.B + 1, cfg.T), dtype=torch.int32), cfg.K, cfg.p, SEED)
