@@ -502,7 +502,8 @@ int dm_enable_js(dm_ctx* c, int max_rows, int max_hidden_rows) {
     c->js_max_rows = c->js_max_hidden = 0;
     const size_t n_logits = (size_t)max_rows * c->head.V * sizeof(float);
     const size_t n_ws = js_workspace_floats(c->head.V, max_rows, max_hidden_rows) * sizeof(float);
-    if (cudaMalloc(&c->js_logits, n_logits) != cudaSuccess || cudaMalloc(&c->js_ws, n_ws) != cudaSuccess) {
+    if (cudaMalloc(&c->js_logits, n_logits) != cudaSuccess || cudaMalloc(&c->js_ws, n_ws) != cudaSuccess ||
+        cudaMemset(c->js_ws, 0, n_ws) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(c->js_logits); c->js_logits = nullptr;
         cudaFree(c->js_ws); c->js_ws = nullptr;
@@ -541,10 +542,11 @@ int dropmatch_verify_js(dm_ctx* c, const void* H, const int32_t* draft, const fl
     fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
     st = run_verify(c, H, (int)rows, map, mk, fa, s, c->js_logits);
     if (st != DM_OK) return st;
-    st = launch_js(c->js_logits, draft_prob, c->js_ws, c->head.V, B, T, K, out_tokens, draft, out_js, out_js_ok,
-                   out_accept_len, c->err, s);
+    st = launch_js(c->js_logits, draft_prob, c->js_ws,
+                   js_workspace_floats(c->head.V, c->js_max_rows, c->js_max_hidden) - 4, c->head.V, B, T, K, out_tokens,
+                   draft, out_js, out_js_ok, out_accept_len, c->err, s);
     if (st != DM_OK) return st;
-    c->last_launches += 3;
+    c->last_launches += K <= 32 ? 2 : 3;
     return DM_OK;
 }
 

@@ -91,11 +91,11 @@ int launch_host_gather(const void* src_h, size_t h_bytes, const int32_t* src_dra
 int launch_read_stream(const void* ptr, size_t bytes, unsigned int* sink, int sms, cudaStream_t stream);
 
 // JS-divergence acceptance (Eq. 4, Eq. 5, Algorithm 1) on logits [B*T*K][V] written by a head kernel.
-int js_chunks(int V);
-size_t js_workspace_floats(int V, int max_rows, int max_hidden);
+int js_chunks(int V, int n_pos);
+size_t js_workspace_floats(int V, int max_rows, int max_hidden);   // the last four floats hold the ticket word (zero)
 constexpr int kJsMaxPositions = 65535;   // B*T of one JS call (a grid dimension)
-int launch_js(const float* logits, const float* draft_prob, float* workspace, int V, int B, int T, int K,
-              const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
+int launch_js(const float* logits, const float* draft_prob, float* workspace, size_t ticket_offset, int V, int B, int T,
+              int K, const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
               int32_t* out_accept_len, const uint32_t* err, cudaStream_t stream);
 
 int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo, int shared_masks,

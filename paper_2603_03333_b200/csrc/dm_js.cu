@@ -123,6 +123,52 @@ js_sum_kernel(const float* __restrict__ logits, const float* __restrict__ draft_
     }
 }
 
+// Algorithm 1 and the left-to-right scan for sequence b, run by one block of kJsThreads threads;
+// also exports the divergences.  `ok` is shared scratch of T ints.
+struct JsAcceptArgs {
+    const float* share;
+    int n_chunks, B, T, K;
+    const int32_t* tokens;
+    const int32_t* draft;
+    float* out_js;
+    int32_t* out_js_ok;
+    int32_t* out_accept_len;
+    const uint32_t* err;
+};
+
+__device__ __forceinline__ void js_accept_sequence(const JsAcceptArgs& a, int b, int32_t* ok) {
+    const int T = a.T, K = a.K, n_chunks = a.n_chunks;
+    // a kernel of this call gave up on a wait: the logits are incomplete, nothing may be accepted
+    const bool failed = a.err != nullptr && *reinterpret_cast<const volatile uint32_t*>(a.err) != 0u;
+    // divergences: one warp per (position, series), lanes over the chunks, summed in double
+    for (int x = threadIdx.x >> 5; x < T * (K + 1); x += kJsThreads / 32) {
+        const size_t idx = (size_t)b * T * (K + 1) + x;
+        double acc = 0.0;
+        for (int c = threadIdx.x & 31; c < n_chunks; c += 32) acc += (double)__ldcg(a.share + idx * n_chunks + c);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+        if ((threadIdx.x & 31) == 0) a.out_js[idx] = (float)acc;
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < T; t += kJsThreads) {
+        const size_t q = (size_t)b * T + t;
+        const float* js = a.out_js + q * (K + 1);
+        float max_heads = js[0];
+        for (int i = 1; i < K; ++i) max_heads = fmaxf(max_heads, js[i]);
+        const bool eq5 = js[K] <= max_heads;                                   // Eq. 5
+        const bool eq6 = position_ok(a.tokens + q * K, K, a.draft[q], DM_RULE_MAJORITY, nullptr);   // Eq. 6
+        if (a.out_js_ok) a.out_js_ok[q] = eq5 && !failed;
+        ok[t] = (eq5 || eq6) && !failed;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int len = 0;
+        while (len < T && ok[len]) ++len;
+        a.out_accept_len[b] = len;
+    }
+    __syncthreads();
+}
+
 // ---- the same two sweeps for K <= KMAX paths with every series kept in registers --------------
 // A thread takes vocabulary entries v0 + tid, v0 + tid + 256, ...: it loads the K logits of an
 // entry once (coalesced across the block), forms the centroid and updates all K+1 running
@@ -185,10 +231,15 @@ js_lse_reg_kernel(const float* __restrict__ logits, int V, int K, int chunk_len,
     }
 }
 
+// The block that finishes last (a ticket counter in global memory, left at zero) also runs
+// Algorithm 1 and the scan for every sequence: no third kernel.
 template <int KMAX>
 __global__ void __launch_bounds__(kJsThreads)
 js_sum_reg_kernel(const float* __restrict__ logits, const float* __restrict__ draft_prob, int V, int K,
-                  int chunk_len, int n_chunks, const float2* __restrict__ part, float* __restrict__ share) {
+                  int chunk_len, int n_chunks, const float2* __restrict__ part, float* __restrict__ share,
+                  unsigned int* __restrict__ ticket, JsAcceptArgs accept) {
+    extern __shared__ int32_t ok_scratch[];   // [T], for the last block
+    __shared__ unsigned int s_ticket;
     __shared__ float lse[KMAX + 1];
     __shared__ float red[kJsThreads / 32][KMAX + 1];
     const int pos = blockIdx.y, chunk = blockIdx.x;
@@ -240,84 +291,72 @@ js_sum_reg_kernel(const float* __restrict__ logits, const float* __restrict__ dr
             share[((size_t)pos * (K + 1) + series) * n_chunks + chunk] = 0.5f * t;
         }
     }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_ticket = atomicAdd(ticket, 1u);
+    __syncthreads();
+    if (s_ticket == gridDim.x * gridDim.y - 1) {
+        __threadfence();
+        for (int b = 0; b < accept.B; ++b) js_accept_sequence(accept, b, ok_scratch);
+        if (threadIdx.x == 0) *ticket = 0u;
+    }
 }
 
-// Algorithm 1 and the left-to-right scan for one sequence; also exports the divergences.
 __global__ void __launch_bounds__(kJsThreads)
-js_accept_kernel(const float* __restrict__ share, int n_chunks, int T, int K, const int32_t* __restrict__ tokens,
-                 const int32_t* __restrict__ draft, float* __restrict__ out_js, int32_t* __restrict__ out_js_ok,
-                 int32_t* __restrict__ out_accept_len, const uint32_t* __restrict__ err) {
+js_accept_kernel(JsAcceptArgs a) {
     extern __shared__ int32_t ok[];   // [T]
-    const int b = blockIdx.x;
-    // a kernel of this call gave up on a wait: the logits are incomplete, nothing may be accepted
-    const bool failed = err != nullptr && *reinterpret_cast<const volatile uint32_t*>(err) != 0u;
-    // divergences: one warp per (position, series), lanes over the chunks, summed in double
-    for (int x = threadIdx.x >> 5; x < T * (K + 1); x += kJsThreads / 32) {
-        const size_t idx = (size_t)b * T * (K + 1) + x;
-        double acc = 0.0;
-        for (int c = threadIdx.x & 31; c < n_chunks; c += 32) acc += (double)share[idx * n_chunks + c];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-        if ((threadIdx.x & 31) == 0) out_js[idx] = (float)acc;
-    }
-    __syncthreads();
-    for (int t = threadIdx.x; t < T; t += kJsThreads) {
-        const size_t q = (size_t)b * T + t;
-        const float* js = out_js + q * (K + 1);
-        float max_heads = js[0];
-        for (int i = 1; i < K; ++i) max_heads = fmaxf(max_heads, js[i]);
-        const bool eq5 = js[K] <= max_heads;                                   // Eq. 5
-        const bool eq6 = position_ok(tokens + q * K, K, draft[q], DM_RULE_MAJORITY, nullptr);   // Eq. 6
-        if (out_js_ok) out_js_ok[q] = eq5 && !failed;
-        ok[t] = (eq5 || eq6) && !failed;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int len = 0;
-        while (len < T && ok[len]) ++len;
-        out_accept_len[b] = len;
-    }
+    js_accept_sequence(a, (int)blockIdx.x, ok);
 }
 
 }  // namespace
 
-int js_chunks(int V) {
-    const int n = (V + 1023) / 1024;   // short chunks: several hundred blocks even for a handful of positions
+// Vocabulary chunks per position.  The two sweeps are short kernels: they must fit the GPU in one
+// wave (four blocks of 256 threads per SM at their register count), so the chunk count follows
+// from the number of positions; chunks of about 1024 entries at most.
+int js_chunks(int V, int n_pos) {
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int n = (V + 1023) / 1024;
+    const int fit = (4 * sms) / (n_pos < 1 ? 1 : n_pos);
+    if (n > fit) n = fit;
     return n < 1 ? 1 : n;
 }
 
 size_t js_workspace_floats(int V, int max_rows, int max_hidden) {
-    // partial (max, sum) pairs and JS shares for every (position, series, chunk)
-    return (size_t)(max_rows + max_hidden) * js_chunks(V) * 3;
+    // partial (max, sum) pairs and JS shares for every (position, series, chunk), at the largest
+    // chunk count; then the ticket word of the second sweep
+    return (size_t)(max_rows + max_hidden) * ((V + 1023) / 1024) * 3 + 4;
 }
 
-int launch_js(const float* logits, const float* draft_prob, float* workspace, int V, int B, int T, int K,
-              const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
+int launch_js(const float* logits, const float* draft_prob, float* workspace, size_t ticket_offset, int V, int B, int T,
+              int K, const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
               int32_t* out_accept_len, const uint32_t* err, cudaStream_t stream) {
-    const int n_pos = B * T, n_chunks = js_chunks(V);
+    const int n_pos = B * T, n_chunks = js_chunks(V, n_pos);
     if (n_pos > kJsMaxPositions) return DM_EUNSUPPORTED;   // positions are the grid's second dimension
     const int chunk_len = (V + n_chunks - 1) / n_chunks;
     float2* part = reinterpret_cast<float2*>(workspace);
     float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
+    unsigned int* ticket = reinterpret_cast<unsigned int*>(workspace + ticket_offset);
     if ((size_t)(K + 1 + chunk_len) * sizeof(float) > 40 * 1024 || (size_t)T * sizeof(int32_t) > 40 * 1024) return DM_EUNSUPPORTED;
     dim3 grid((unsigned)n_chunks, (unsigned)n_pos);
+    const JsAcceptArgs acc{share, n_chunks, B, T, K, tokens, draft, out_js, out_js_ok, out_accept_len, err};
+    const size_t ok_bytes = (size_t)T * sizeof(int32_t);
     if (K <= 8) {
         js_lse_reg_kernel<8><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_reg_kernel<8><<<grid, kJsThreads, 0, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share);
+        js_sum_reg_kernel<8><<<grid, kJsThreads, ok_bytes, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share, ticket, acc);
     } else if (K <= 16) {
         js_lse_reg_kernel<16><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_reg_kernel<16><<<grid, kJsThreads, 0, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share);
+        js_sum_reg_kernel<16><<<grid, kJsThreads, ok_bytes, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share, ticket, acc);
     } else if (K <= 32) {
         js_lse_reg_kernel<32><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_reg_kernel<32><<<grid, kJsThreads, 0, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share);
-    } else {   // more paths than fit in registers: one series at a time
+        js_sum_reg_kernel<32><<<grid, kJsThreads, ok_bytes, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share, ticket, acc);
+    } else {   // more paths than fit in registers: one series at a time, acceptance in a kernel of its own
         js_lse_kernel<<<grid, kJsThreads, chunk_len * sizeof(float), stream>>>(logits, V, K, chunk_len, n_chunks, part);
         js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K,
                                                                                       chunk_len, n_chunks, part, share);
+        if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
+        js_accept_kernel<<<B, kJsThreads, ok_bytes, stream>>>(acc);
     }
-    if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
-    js_accept_kernel<<<B, kJsThreads, T * sizeof(int32_t), stream>>>(share, n_chunks, T, K, tokens, draft, out_js,
-                                                                  out_js_ok, out_accept_len, err);
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 
