@@ -83,6 +83,14 @@ int dm_destroy(dm_ctx* ctx);
  * beyond).  Synchronises the device (re-allocation); pins host memory for the *_host call. */
 int dm_set_head(dm_ctx* ctx, const void* W, int V, int d, int dtype, int max_rows, int max_hidden_rows);
 
+/* Programmatic stream serialization of the tensor-core kernel, on by default: the kernel starts
+ * streaming W while the kernel ahead of it in the stream is still finishing, which is only right
+ * if nothing ahead in the stream writes W.  A caller that refreshes W in stream order (a weight
+ * reload, a dequantisation into the head buffer) and verifies right behind it on the same stream
+ * switches it off with dm_set_pdl(ctx, 0): every verify kernel then starts after all earlier work
+ * of the stream has completed, at the cost of about 2 us of launch latency per call. */
+int dm_set_pdl(dm_ctx* ctx, int enable);
+
 /* Force a kernel family (DM_IMPL_*) for later calls; DM_IMPL_AUTO restores the default choice.
  * DM_IMPL_TCGEN05 on a head it cannot handle makes verify calls return DM_EUNSUPPORTED. */
 int dm_set_impl(dm_ctx* ctx, int impl);
@@ -225,7 +233,11 @@ int dropmatch_finalize_packed(dm_ctx* ctx, const uint64_t* packed, int n_parts, 
  * Limits and rules:
  *   - B*T*K <= DM_STATIC_MAX_ROWS, else DM_ESTATICLIMIT and nothing is launched.
  *   - The first call on a device looks the array's device address up (once per device and
- *     process).  Make that first call before any stream capture begins.
+ *     process).  With CUDA's lazy module loading that first call is also when the driver loads
+ *     the code and sets the 0.6 MB array aside, which can fail (DM_ECUDA) once a pool owns all
+ *     of the device's memory: make one call per device at start-up, before the pool takes the
+ *     memory and before any stream capture begins.  The remembered address does not survive a
+ *     cudaDeviceReset.
  *   - All calls on a device share the one array, which keeps the previous call's contents; the
  *     call itself clears the part that must start at zero.  Two calls whose kernels can overlap
  *     on the GPU (different streams, or host threads racing on one device) corrupt each other:

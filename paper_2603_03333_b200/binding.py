@@ -29,6 +29,7 @@ SIGNATURES = {
     "dm_destroy": (_ci, [_vp]),
     "dm_set_head": (_ci, [_vp, _vp, _ci, _ci, _ci, _ci, _ci]),
     "dm_set_impl": (_ci, [_vp, _ci]),
+    "dm_set_pdl": (_ci, [_vp, _ci]),
     "dm_set_mask_mode": (_ci, [_vp, _ci]),
     "dm_set_vocab_offset": (_ci, [_vp, _ci]),
     "dropmatch_partial_best": (_ci, [_vp, _vp, _ci, _ci, _ci, _cf, _u64, _u64, _vp, _vp]),
@@ -153,6 +154,8 @@ class Context:
 
     # -- dm_set_head / dm_set_impl
     def set_head(self, W: torch.Tensor, max_rows: int, max_hidden_rows: int | None = None):
+        """W must be complete before a verify call is enqueued and must not be written by work that
+        is still in flight on the stream (see set_pdl)."""
         if W.dtype not in (torch.float32, torch.bfloat16) or not W.is_cuda or not W.is_contiguous() or W.dim() != 2:
             raise TypeError("W must be a contiguous 2-D CUDA tensor of float32 or bfloat16")
         dtype = F32 if W.dtype == torch.float32 else BF16
@@ -162,6 +165,11 @@ class Context:
 
     def set_impl(self, impl: int):
         _check(lib().dm_set_impl(self._h, impl), "dm_set_impl")
+
+    def set_pdl(self, enable: bool):
+        """Off: verify kernels never start before earlier work of the stream has completed (needed when
+        that work writes W; by default the kernel streams W while the kernel ahead is still finishing)."""
+        _check(lib().dm_set_pdl(self._h, int(enable)), "dm_set_pdl")
 
     def set_mask_mode(self, mode: int):
         _check(lib().dm_set_mask_mode(self._h, mode), "dm_set_mask_mode")

@@ -15,6 +15,7 @@ struct dm_ctx {
     int max_rows = 0, max_hidden = 0;
     int impl = DM_IMPL_AUTO;
     int mask_mode = DM_MASK_PER_POSITION;
+    bool pdl = true;                         // head kernel launched with programmatic stream serialization (dm_set_pdl)
     long long wait_limit = 0;                // clock cycles a kernel waits on a barrier before it gives up; 0 = default
     int last_impl = 0, last_launches = 0;
     // workspace (device)
@@ -143,7 +144,7 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
                           logits_out, c->err, stream, &launches, &fa, c->err + 1,
-                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded, nullptr, c->wait_limit);
+                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded, nullptr, c->wait_limit, c->pdl);
     else {
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, logits_out, c->err, stream);
         launches = 1;
@@ -303,7 +304,7 @@ int dropmatch_partial_best(dm_ctx* c, const void* H, int B, int T, int K, float 
             return DM_ECUDA;
         }
         st = fused_launch(c->fused, c->head, H, B * T, rows, map, mk, &n_slices, c->partials, nullptr, c->err, s,
-                          &launches, nullptr, nullptr, nullptr, &reduced, out, c->wait_limit);
+                          &launches, nullptr, nullptr, nullptr, &reduced, out, c->wait_limit, c->pdl);
     } else {
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, nullptr, c->err, s);
     }
@@ -337,6 +338,12 @@ int dropmatch_finalize_packed(dm_ctx* c, const uint64_t* packed, int n_parts, co
     fa.err = c->err;
     return launch_finalize(reinterpret_cast<const unsigned long long*>(packed), n_parts, B * T * K, fa,
                            static_cast<cudaStream_t>(stream));
+}
+
+int dm_set_pdl(dm_ctx* c, int enable) {
+    if (c == nullptr) return DM_EINVAL;
+    c->pdl = enable != 0;
+    return DM_OK;
 }
 
 int dm_debug_set_wait_limit(dm_ctx* c, uint64_t cycles) {

@@ -72,6 +72,10 @@ struct FusedParams {
     int group_tiles;  // tiles whose accumulators are live together
     int n_slots;      // accumulator slots in TMEM (512 / n_pad)
     int nsw, nsb;     // stages of the W ring and of the operand ring
+    // staged: one ring of `nsw` steps.  A step holds the group's W tiles of one hidden-size block and,
+    // behind them, the operand block; one barrier says that all of it has landed, one that the MMAs
+    // are done with it, so that the issuing thread waits and commits once per step.
+    uint32_t step_bytes;
     int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
     int pdl;          // launched with programmatic stream serialization: see the griddep_wait() calls
     long long wait_limit;   // clock cycles after which a wait on an mbarrier gives up (see dm_debug_set_wait_limit)
@@ -148,7 +152,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     if (threadIdx.x == 0) {
         ptx::prefetch_tensormap(&tmap_w);
         if (P.staged) ptx::prefetch_tensormap(&tmap_b);
-        for (int s = 0; s < P.nsw; ++s) { ptx::mbar_init(w_full + 8 * s, 1); ptx::mbar_init(w_empty + 8 * s, 1); }
+        for (int s = 0; s < P.nsw; ++s) { ptx::mbar_init(w_full + 8 * s, P.staged ? 2 : 1); ptx::mbar_init(w_empty + 8 * s, 1); }
         for (int s = 0; s < P.nsb; ++s) {
             ptx::mbar_init(b_ready + 8 * s, P.staged ? 1 : wps);
             ptx::mbar_init(b_empty + 8 * s, 1);
@@ -209,6 +213,34 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         const uint32_t tx_bytes = (uint32_t)P.tile_rows * (kBlockK * 2);
         uint32_t bar_full = w_full, bar_empty = w_empty, dst = smem_base + P.off_w, empty_parity = 1;
         int stage = 0;
+        if (P.staged) {
+            // one step per (group, hidden-size block): the group's W tiles side by side
+            for (int g = 0; g < n_groups; ++g) {
+                const int t0 = g * G, t1 = min(my_tiles, t0 + G);
+                const int v_first = v_cta0 + t0 * P.tile_rows;
+                const uint32_t step_tx = (uint32_t)(t1 - t0) * tx_bytes;
+                for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
+                    if (!ptx::mbar_wait<kPollNs>(bar_empty, empty_parity, s_abort, P.wait_limit)) {
+                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_EMPTY);
+                        return;
+                    }
+                    if (!kPair) ptx::mbar_arrive_expect_tx(bar_full, step_tx);
+                    else if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full, 2 * step_tx);   // both CTAs' tiles count here
+                    int v_tile = v_first;
+                    uint32_t d = dst;
+                    for (int tile = t0; tile < t1; ++tile, v_tile += P.tile_rows, d += kWStageBytes) {
+                        if (kPair) ptx::tma_load_2d_pair(d, &tmap_w, x, v_tile, ptx::map_to_cta(bar_full, 0));
+                        else ptx::tma_load_2d(d, &tmap_w, x, v_tile, bar_full);
+                    }
+                    bar_full += 8; bar_empty += 8; dst += P.step_bytes;
+                    if (++stage == P.nsw) {
+                        stage = 0; empty_parity ^= 1;
+                        bar_full = w_full; bar_empty = w_empty; dst = smem_base + P.off_w;
+                    }
+                }
+            }
+            return;
+        }
         for (int g = 0; g < n_groups; ++g) {
             const int t0 = g * G, t1 = min(my_tiles, t0 + G);
             const int v_first = v_cta0 + t0 * P.tile_rows;
@@ -238,7 +270,10 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     }
     if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane != 0 || rank != 0) return;
+        // The whole warp runs the loops below converged and one elected lane issues the MMAs and the
+        // commits: every value an MMA takes then lives in uniform registers (a lone surviving lane
+        // would pay a register move per operand, and the issuing thread is the busiest of the CTA).
+        if (rank != 0) return;
         const uint32_t idesc = ptx::idesc_bf16_f32(kPair ? 2 * kTileM : kTileM, P.n_pad);
         const uint32_t b_stage_bytes = (uint32_t)(kPair ? P.n_pad / 2 : P.n_pad) * (kBlockK * 2);
         const uint64_t a_desc0 = ptx::smem_desc_sw128(smem_base + P.off_w);
@@ -248,49 +283,109 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         uint32_t w_parity = 0, b_parity = 0, slot_parity = 1;   // slot_parity: parity of the slot_empty wait
         uint64_t a_desc = a_desc0, b_desc = b_desc0;
         uint32_t bar_wf = w_full, bar_we = w_empty, bar_br = b_ready, bar_be = b_empty;
+        if (P.staged) {
+            // One wait and one commit per step: the step's barrier covers its W tiles and its operand
+            // block.  The whole warp runs this loop converged and one elected lane issues: every
+            // value an MMA takes then lives in uniform registers.
+            const uint32_t step_units = P.step_bytes >> 4;
+            b_desc = ptx::smem_desc_sw128(smem_base + P.off_w + (uint32_t)G * kWStageBytes);
+            const uint64_t b_step0 = b_desc;
+            for (int g = 0; g < n_groups; ++g) {
+                const int t0 = g * G, t1 = min(my_tiles, t0 + G);
+                const int slot0 = slot;
+                for (int tile = t0; tile < t1; ++tile) {   // the group's accumulator slots must be drained
+                    if (!ptx::mbar_wait_converged<kPollNs, true>(slot_empty + 8 * slot, slot_parity, s_abort, P.wait_limit)) {
+                        if (lane == 0) atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
+                        return;
+                    }
+                    if (++slot == P.n_slots) { slot = 0; slot_parity ^= 1; }
+                }
+                ptx::tc_fence_after();
+                for (int kb = 0; kb < P.kb_count; ++kb) {
+                    if (!ptx::mbar_wait_converged<kPollNs, true>(bar_wf, w_parity, s_abort, P.wait_limit)) {
+                        if (lane == 0) atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
+                        return;
+                    }
+                    ptx::tc_fence_after();
+                    if (ptx::elect_one()) {
+                        int sl = slot0;
+                        uint32_t d_tmem = tmem_base + (uint32_t)(slot0 * P.n_pad);
+                        uint64_t a_tile = a_desc;
+                        for (int tile = t0; tile < t1; ++tile) {
+#pragma unroll
+                            for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
+                                if (kPair) ptx::mma_f16_pair(d_tmem, a_tile + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                                else ptx::mma_f16(d_tmem, a_tile + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                            a_tile += kWStageBytes >> 4;
+                            d_tmem += (uint32_t)P.n_pad;
+                            if (++sl == P.n_slots) { sl = 0; d_tmem = tmem_base; }
+                        }
+                        if (kPair) ptx::mma_commit_pair(bar_we, 3); else ptx::mma_commit(bar_we);
+                    }
+                    __syncwarp();
+                    bar_wf += 8; bar_we += 8; a_desc += step_units; b_desc += step_units;
+                    if (++sw == P.nsw) { sw = 0; w_parity ^= 1; bar_wf = w_full; bar_we = w_empty; a_desc = a_desc0; b_desc = b_step0; }
+                }
+                if (ptx::elect_one()) {
+                    int sl = slot0;
+                    for (int tile = t0; tile < t1; ++tile) {
+                        if (kPair) ptx::mma_commit_pair(slot_full + 8 * sl, 3); else ptx::mma_commit(slot_full + 8 * sl);
+                        if (++sl == P.n_slots) sl = 0;
+                    }
+                }
+                __syncwarp();
+            }
+            return;
+        }
         for (int g = 0; g < n_groups; ++g) {
             const int t0 = g * G, t1 = min(my_tiles, t0 + G);
             const int slot0 = slot;
             for (int tile = t0; tile < t1; ++tile) {   // the group's accumulator slots must be drained
-                if (!ptx::mbar_wait<kPollNs>(slot_empty + 8 * slot, slot_parity, s_abort, P.wait_limit)) {
-                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
+                if (!ptx::mbar_wait_converged<kPollNs, false>(slot_empty + 8 * slot, slot_parity, s_abort, P.wait_limit)) {
+                    if (lane == 0) atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_ACC_EMPTY);
                     return;
                 }
                 if (++slot == P.n_slots) { slot = 0; slot_parity ^= 1; }
             }
             ptx::tc_fence_after();
             for (int kb = 0; kb < P.kb_count; ++kb) {
-                if (!ptx::mbar_wait<kPollNs>(bar_br, b_parity, s_abort, P.wait_limit)) {
-                    atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
+                if (!ptx::mbar_wait_converged<kPollNs, false>(bar_br, b_parity, s_abort, P.wait_limit)) {
+                    if (lane == 0) atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_OPERAND);
                     return;
                 }
                 int sl = slot0;
                 uint32_t d_tmem = tmem_base + (uint32_t)(slot0 * P.n_pad);
                 for (int tile = t0; tile < t1; ++tile) {
-                    if (!ptx::mbar_wait<kPollNs>(bar_wf, w_parity, s_abort, P.wait_limit)) {
-                        atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
+                    if (!ptx::mbar_wait_converged<kPollNs, false>(bar_wf, w_parity, s_abort, P.wait_limit)) {
+                        if (lane == 0) atomicCAS(P.err, 0u, (uint32_t)ERR_WAIT_FULL);
                         return;
                     }
                     ptx::tc_fence_after();
+                    if (ptx::elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
-                        if (kPair) ptx::mma_f16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-                        else ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-                    if (kPair) ptx::mma_commit_pair(bar_we, 3); else ptx::mma_commit(bar_we);
+                        for (int k = 0; k < kBlockK / 16; ++k)   // 16 elements = 32 bytes = 2 descriptor units
+                            ptx::mma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                        ptx::mma_commit(bar_we);
+                    }
+                    __syncwarp();
                     bar_wf += 8; bar_we += 8; a_desc += kWStageBytes >> 4;
                     if (++sw == P.nsw) { sw = 0; w_parity ^= 1; bar_wf = w_full; bar_we = w_empty; a_desc = a_desc0; }
                     d_tmem += (uint32_t)P.n_pad;
                     if (++sl == P.n_slots) { sl = 0; d_tmem = tmem_base; }
                 }
-                if (kPair) ptx::mma_commit_pair(bar_be, 3); else ptx::mma_commit(bar_be);
+                if (ptx::elect_one()) ptx::mma_commit(bar_be);
+                __syncwarp();
                 bar_br += 8; bar_be += 8; b_desc += b_stage_bytes >> 4;
                 if (++sb == P.nsb) { sb = 0; b_parity ^= 1; bar_br = b_ready; bar_be = b_empty; b_desc = b_desc0; }
             }
-            int sl = slot0;
-            for (int tile = t0; tile < t1; ++tile) {
-                if (kPair) ptx::mma_commit_pair(slot_full + 8 * sl, 3); else ptx::mma_commit(slot_full + 8 * sl);
-                if (++sl == P.n_slots) sl = 0;
+            if (ptx::elect_one()) {
+                int sl = slot0;
+                for (int tile = t0; tile < t1; ++tile) {
+                    ptx::mma_commit(slot_full + 8 * sl);
+                    if (++sl == P.n_slots) sl = 0;
+                }
             }
+            __syncwarp();
         }
         return;
     }
@@ -306,7 +401,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             const int b_rows = kPair ? P.n_pad / 2 : P.n_pad;      // a pair splits the operand rows
             const int b_row0 = row0 + (int)rank * b_rows;
             const uint32_t b_stage_bytes = (uint32_t)b_rows * (kBlockK * 2);
-            uint32_t bar_r = b_ready, bar_e = b_empty, dst = smem_base + P.off_b, parity = 1;
+            // the operand block of a step lands behind the step's W tiles and counts on the same barrier
+            const uint32_t dst0 = smem_base + P.off_w + (uint32_t)G * kWStageBytes;
+            uint32_t bar_r = w_full, bar_e = w_empty, dst = dst0, parity = 1;
             int stage = 0;
             for (int g = 0; g < n_groups; ++g)
                 for (int kb = 0, x = 0; kb < P.kb_count; ++kb, x += kBlockK) {
@@ -321,8 +418,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                         ptx::mbar_arrive_expect_tx(bar_r, b_stage_bytes);
                         ptx::tma_load_2d(dst, &tmap_b, x, b_row0, bar_r);
                     }
-                    bar_r += 8; bar_e += 8; dst += b_stage_bytes;
-                    if (++stage == P.nsb) { stage = 0; parity ^= 1; bar_r = b_ready; bar_e = b_empty; dst = smem_base + P.off_b; }
+                    bar_r += 8; bar_e += 8; dst += P.step_bytes;
+                    if (++stage == P.nsw) { stage = 0; parity ^= 1; bar_r = w_full; bar_e = w_empty; dst = dst0; }
                 }
             return;
         }
@@ -671,11 +768,16 @@ struct SmemPlan {
     int nsw, nsb, group_tiles, n_slots, staged;
     int pair;    // run as clusters of two CTAs that split the operand rows
     int n_pad;   // operand rows after padding: a multiple of 16, of 32 for pairs
+    uint32_t step_bytes;   // staged: bytes of one step (the group's W tiles, then the operand block)
     uint32_t off_w, off_b, off_rowinfo, off_best, off_bar, total;
 };
 
+#ifndef DM_EXPOSE_SLOTS
+#define DM_EXPOSE_SLOTS 0
+#endif
+
 // Choose the operand mode (builders, staged, staged as CTA pairs) and the tile grouping, then
-// split the 227 KB of shared memory between the W ring and the operand ring.
+// split the 227 KB of shared memory between the rings.
 bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     SmemPlan best{};
     int n_pad = (rows + 15) & ~15;
@@ -694,38 +796,42 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
         best.group_tiles = tiles_per_cta;
         best.staged = 0;
         best.nsb = 4;
+        for (;;) {   // shrink the operand ring until the W ring has six stages (or the ring is at two)
+            const uint32_t used = (uint32_t)best.nsb * b_stage;
+            if (used + 2u * kWStageBytes <= avail) {
+                best.nsw = (int)((avail - used) / kWStageBytes);
+                if (best.nsw > kMaxWStages) best.nsw = kMaxWStages;
+                if (best.nsw >= 6 || best.nsb == 2) break;
+            }
+            if (best.nsb == 2) return false;
+            best.nsb = 2;   // the eight builder warps split evenly over 4 or 2 stages
+        }
+        best.off_w = 0;
+        best.off_b = (uint32_t)best.nsw * kWStageBytes;
+        best.off_rowinfo = best.off_b + (uint32_t)best.nsb * b_stage;
     } else {
         // Several groups: the operand would have to be rebuilt for every group, so it is staged
         // through global memory by mask_operand_kernel and streamed in by TMA (no builders).
-        // With four or more slots a group takes half of them, so that the epilogue of one group
-        // overlaps the MMAs of the next; with fewer, a group takes them all, which halves the
-        // operand traffic and leaves the epilogue exposed.  Group sizes are evened out.
-        int g = best.n_slots >= 4 ? best.n_slots / 2 : best.n_slots;
+        // A group takes at most half of the accumulator slots, so that the epilogue of one group
+        // overlaps the MMAs of the next (with two or three slots: single tiles).  The operand is
+        // then fetched once per group, from L2, which costs nothing measurable: halving or
+        // quartering those loads left the kernel's time unchanged.  Group sizes are evened out.
+        int g = best.n_slots / 2;
+        if (g < 1) g = 1;
+        if (best.n_slots <= DM_EXPOSE_SLOTS) g = best.n_slots;
         const int n_groups = (tiles_per_cta + g - 1) / g;
         best.group_tiles = (tiles_per_cta + n_groups - 1) / n_groups;
         best.staged = 1;
-        // operand ring: up to 96 KB in two to eight stages.  Its blocks come from L2 with a
-        // latency of a few microseconds under load and a stage lasts only group_tiles W steps,
-        // so the ring has to be deep, not large.
-        // Pairs (half-height blocks) afford up to eight stages; a lone CTA keeps four at most,
-        // its W ring needs the room more.
-        best.nsb = (int)(96u * 1024u / b_stage);
-        if (best.nsb > (best.pair ? 8 : 4)) best.nsb = best.pair ? 8 : 4;
-        if (best.nsb < 2) best.nsb = 2;
+        // One ring of steps; a step = the group's W tiles of one hidden-size block + the operand block.
+        best.step_bytes = (uint32_t)best.group_tiles * kWStageBytes + b_stage;
+        best.nsw = (int)(avail / best.step_bytes);
+        if (best.nsw > kMaxWStages) best.nsw = kMaxWStages;
+        if (best.nsw < 2) return false;
+        best.nsb = 1;   // no separate operand ring
+        best.off_w = 0;
+        best.off_b = 0;
+        best.off_rowinfo = (uint32_t)best.nsw * best.step_bytes;
     }
-    for (;;) {   // shrink the operand ring until the W ring has six stages (or the ring is at two)
-        const uint32_t used = (uint32_t)best.nsb * b_stage;
-        if (used + 2u * kWStageBytes <= avail) {
-            best.nsw = (int)((avail - used) / kWStageBytes);
-            if (best.nsw > kMaxWStages) best.nsw = kMaxWStages;
-            if (best.nsw >= 6 || best.nsb == 2) break;
-        }
-        if (best.nsb == 2) return false;
-        best.nsb = best.staged ? best.nsb - 1 : 2;   // the eight builder warps split evenly over 4 or 2 stages
-    }
-    best.off_w = 0;
-    best.off_b = (uint32_t)best.nsw * kWStageBytes;
-    best.off_rowinfo = best.off_b + (uint32_t)best.nsb * b_stage;
     best.off_best = best.off_rowinfo + 256u * sizeof(RowInfo);
     best.off_bar = best.off_best + 4u * n_pad * 8u;
     best.total = best.off_bar + kBarBytes + 1024u;
@@ -831,7 +937,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out,
-                 unsigned long long* packed_out, long long wait_limit) {
+                 unsigned long long* packed_out, long long wait_limit, bool allow_pdl) {
     if (folded_out) *folded_out = false;
     if (fs == nullptr || !fused_supported(head, rows) || fs->geo[0].n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
     // Slices of one-block launches: an even count (pairs need one); a CTA whose slice lies past the
@@ -881,7 +987,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.kb_count = head.d / kBlockK;
         P.tiles_per_cta = geo.tiles_per_cta; P.tile_rows = geo.tile_rows; P.slice_rows = geo.slice_rows;
         P.group_tiles = plan.group_tiles; P.n_slots = plan.n_slots;
-        P.nsw = plan.nsw; P.nsb = plan.nsb; P.staged = plan.staged;
+        P.nsw = plan.nsw; P.nsb = plan.nsb; P.staged = plan.staged; P.step_bytes = plan.step_bytes;
         if (plan.staged && !operand_staged) {
             // one pass over all rows of the call; the launches below read their own rows of it
             if (fs->staging == nullptr || rows > fs->staging_rows) return DM_EWORKSPACE;
@@ -913,7 +1019,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         }
         // Programmatic stream serialization, except when the row selection of the debug call could
         // itself be the output of the kernel ahead (it is read in the prologue).
-        P.pdl = map.sel == nullptr ? 1 : 0;
+        P.pdl = (map.sel == nullptr && allow_pdl) ? 1 : 0;
         P.wait_limit = wait_limit > 0 ? wait_limit : kWaitLimitCycles;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)grid);

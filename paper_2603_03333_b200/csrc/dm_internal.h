@@ -78,7 +78,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidd
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
                  unsigned long long* best = nullptr, bool* folded_out = nullptr,
-                 unsigned long long* packed_out = nullptr, long long wait_limit = 0);
+                 unsigned long long* packed_out = nullptr, long long wait_limit = 0, bool allow_pdl = true);
 
 // The staged masked operand of the tensor-core kernel (Eq. 1 and the numerator of Eq. 2), written to `out`.
 int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,

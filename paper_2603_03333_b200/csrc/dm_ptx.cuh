@@ -69,6 +69,56 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 
+// The same wait for a warp that must stay converged: every lane runs the loop and every branch
+// in it depends on a warp-wide value only.  For the warp that issues the tcgen05 instructions:
+// their operands live in uniform registers, which the compiler can only use while the warp is
+// converged and the values do not depend on the lane; a lone surviving lane pays a register move
+// per operand.  ALL_LANES: every lane polls (one instruction for the warp, one barrier word) and
+// a vote decides, the quickest way out when the wait is short and on the critical path;
+// otherwise lane 0 polls and broadcasts, which disturbs the TMA unit least when the warp mostly
+// waits.
+template <int SLEEP_NS, bool ALL_LANES>
+__device__ __forceinline__ bool mbar_wait_converged(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                    long long limit_cycles) {
+    if (ALL_LANES) {
+        if (__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) return true;
+        const long long t0 = clock64();
+        for (;;) {
+            if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+            if (__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) return true;
+            const bool give_up = *abort_flag != 0 || clock64() - t0 > limit_cycles;
+            if (__any_sync(0xFFFFFFFFu, give_up)) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    const bool poller = (threadIdx.x & 31) == 0;
+    long long t0 = 0;
+    for (int tries = 0;; ++tries) {
+        int state = 0;   // 1: phase complete, 2: give up
+        if (poller) {
+            if (mbar_try_wait(bar, parity)) state = 1;
+            else if (*abort_flag) state = 2;
+            else if (tries == 1) t0 = clock64();
+            else if (tries > 1 && clock64() - t0 > limit_cycles) { *abort_flag = 1; state = 2; }
+        }
+        state = __shfl_sync(0xFFFFFFFFu, state, 0);
+        if (state != 0) return state == 1;
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+    }
+}
+// One lane of a converged warp, the same one every time.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xFFFFFFFF;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // ---- TMA ----------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");

@@ -420,3 +420,27 @@ def test_tree_with_plain_tokens(ctx):
             assert np.array_equal(got[key], base[key]), key
         bad = (got["plain"] != plain_ref["plain"]) & (plain_ref["plain_gap"] >= NEAR_TIE)
         assert not bad.any()
+
+
+def test_head_rewritten_in_stream_order_with_pdl_off(ctx):
+    """A caller that refreshes W on the stream right before it verifies (a weight reload, a
+    dequantisation into the head buffer) switches programmatic stream serialization off: the
+    verify kernel then starts only after the write has completed.  Refereed by the oracle on the
+    new head."""
+    cfg = wl.Config("reload", d=512, V=30000, dtype=wl.BF16, B=2, T=3, K=8, p=0.1)
+    work = wl.make_workload(cfg, device=DEV)
+    W_new = wl.make_head(cfg.V, cfg.d, cfg.dtype, seed=77, device=DEV)
+    W_buf = work.W.clone()
+    ctx.set_head(W_buf, max_rows=cfg.rows)
+    ctx.set_pdl(False)
+    try:
+        ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED)       # a call on the old head is in flight
+        W_buf.copy_(W_new)                                               # ... the head is rewritten on the same stream
+        got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))   # ... and used right behind it
+        assert ctx.device_error() == 0
+    finally:
+        ctx.set_pdl(True)
+    draft = work.draft.cpu().numpy()
+    ref = oracle.verify_batched(wl.to_numpy_storage(W_new), cfg.dtype, wl.to_numpy_storage(work.H), draft, cfg.K,
+                                cfg.p, SEED)
+    check_chain(got, ref, draft)
