@@ -44,10 +44,7 @@ int launch_merge_partials(const unsigned long long* partials, int n_slices, int 
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 
-size_t finalize_smem_bytes(int T, int K, int N) {
-    size_t extra = N > 0 ? 2 * (size_t)N : (size_t)T;
-    return ((size_t)T * K + extra) * sizeof(int32_t);
-}
+size_t finalize_smem_bytes(int T, int K, int N) { return finalize_smem_bytes_dev(T, K, N); }
 
 int launch_finalize(const unsigned long long* partials, int n_slices, int rows,
                     const FinalizeArgs& a, cudaStream_t stream) {

@@ -7,6 +7,12 @@
 
 namespace dm {
 
+// Bytes of scratch finalize_sequence needs (the host's finalize_smem_bytes, for device code).
+__host__ __device__ __forceinline__ size_t finalize_smem_bytes_dev(int T, int K, int N) {
+    const size_t extra = N > 0 ? 2 * (size_t)N : (size_t)T;
+    return ((size_t)T * K + extra) * sizeof(int32_t);
+}
+
 struct BlockSync {
     __device__ __forceinline__ void operator()() const { __syncthreads(); }
 };
@@ -16,6 +22,11 @@ struct NamedSync {
     __device__ __forceinline__ void operator()() const {
         asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
     }
+};
+
+// __syncwarp: one warp runs finalize_sequence on its own (nthreads = 32).
+struct WarpSync {
+    __device__ __forceinline__ void operator()() const { __syncwarp(); }
 };
 
 // Does `draft` pass `rule` against the K tokens of one hidden row (shared memory)?

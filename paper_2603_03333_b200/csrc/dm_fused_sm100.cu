@@ -55,7 +55,10 @@ constexpr int kIdlePollNs = 500;            // ... and of one that completes onc
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort flag
 #ifndef DM_PAIR_MIN_NPAD
-#define DM_PAIR_MIN_NPAD 176
+#define DM_PAIR_MIN_NPAD 64
+#endif
+#ifndef DM_STAGED_MIN_NPAD
+#define DM_STAGED_MIN_NPAD 64   // launches at least this wide are staged even if the slice would fit TMEM as one group
 #endif
 constexpr int kPairMinNPad = DM_PAIR_MIN_NPAD;   // staged launches at least this wide run as CTA pairs
 
@@ -689,9 +692,22 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             ptx::bar_sync(1, 4 * 32);
             if (*s_ticket == gridDim.x - 1) {
                 __threadfence();
-                int32_t* scratch = reinterpret_cast<int32_t*>(smem + P.off_w);   // the W ring is idle by now
-                for (int b = 0; b < P.fin.B; ++b)
-                    finalize_sequence(P.best, 1, P.rows_total, P.fin, b, scratch, tid_e, 4 * 32, NamedSync{1, 4 * 32});
+                int32_t* scratch = reinterpret_cast<int32_t*>(smem + P.off_w);   // the rings are idle by now
+                if (P.fin.B == 1) {
+                    finalize_sequence(P.best, 1, P.rows_total, P.fin, 0, scratch, tid_e, 4 * 32, NamedSync{1, 4 * 32});
+                } else {
+                    // several sequences: each warp takes its own (a sequence is a chain of dependent
+                    // global accesses of about 10 us; four of them run side by side), with scratch
+                    // of its own if the idle rings have room for it
+                    const uint32_t need = ((uint32_t)finalize_smem_bytes_dev(P.fin.T, P.fin.K + P.fin.plain, P.fin.N) + 15u) & ~15u;
+                    const int n_par = min(4, (int)(P.off_rowinfo / need));
+                    const int w = warp - kFirstEpiWarp;
+                    if (w < n_par)
+                        for (int b = w; b < P.fin.B; b += n_par)
+                            finalize_sequence(P.best, 1, P.rows_total, P.fin, b, scratch + (size_t)w * (need / 4), lane, 32,
+                                              WarpSync{});
+                    ptx::bar_sync(1, 4 * 32);
+                }
                 for (int n = tid_e; n < P.rows_total; n += 4 * 32) P.best[n] = 0ull;   // ready for the next call
                 if (tid_e == 0) *P.ticket = 0u;
             }
@@ -706,6 +722,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 __global__ void __launch_bounds__(256)
 mask_operand_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat16* __restrict__ out, int rows, int d,
                     RowMap map, uint32_t key0, uint32_t key1, uint32_t thr, uint32_t* __restrict__ err) {
+    // The head kernel behind this one may be scheduled at once: it streams W until its operand
+    // producer needs these rows, and that thread waits for this kernel to finish.
+    ptx::griddep_launch_dependents();
     const int chunks = d >> 3;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)rows * chunks) return;
@@ -783,14 +802,15 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     int n_pad = (rows + 15) & ~15;
     // Staged launches with many operand rows run as CTA pairs: at N >= kPairMinNPad the operand
     // reads of a lone CTA's MMAs, added to the TMA writes, saturate its shared memory.
-    best.pair = (tiles_per_cta > kTmemCols / n_pad && n_pad >= kPairMinNPad) ? 1 : 0;
+    const bool force_staged = n_pad >= DM_STAGED_MIN_NPAD && tiles_per_cta > 1;
+    best.pair = ((tiles_per_cta > kTmemCols / n_pad || force_staged) && n_pad >= kPairMinNPad) ? 1 : 0;
     if (best.pair) n_pad = (rows + 31) & ~31;
     best.n_pad = n_pad;
     best.n_slots = kTmemCols / n_pad;
     const uint32_t b_stage = (uint32_t)(best.pair ? n_pad / 2 : n_pad) * (kBlockK * 2);
     const uint32_t fixed = 256u * sizeof(RowInfo) + 4u * n_pad * 8u + kBarBytes;
     const uint32_t avail = kSmemLimit - 1024 - fixed;
-    if (tiles_per_cta <= best.n_slots) {
+    if (tiles_per_cta <= best.n_slots && !force_staged) {
         // One group: the whole slice is live at once and the builders generate the masks in
         // registers, once per call.  Four small operand stages, the rest goes to the W ring.
         best.group_tiles = tiles_per_cta;
@@ -819,6 +839,7 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
         int g = best.n_slots / 2;
         if (g < 1) g = 1;
         if (best.n_slots <= DM_EXPOSE_SLOTS) g = best.n_slots;
+        if (g >= tiles_per_cta) g = (tiles_per_cta + 1) / 2;   // at least two groups: the first epilogue overlaps
         const int n_groups = (tiles_per_cta + g - 1) / g;
         best.group_tiles = (tiles_per_cta + n_groups - 1) / n_groups;
         best.staged = 1;
