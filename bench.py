@@ -30,7 +30,8 @@ WORKLOAD = "llama8b"   # Llama-3-8B-shaped head: the configuration the metric is
 
 # DRAM bytes (read + write) of one fused head-kernel launch on this workload, from the ncu capture
 # summarised in profiles/; None until a capture exists.
-NCU_TRAFFIC_BYTES = {"llama8b": 1051084000 + 4251000, "llama8b_k32": 1059248000 + 5305000}
+NCU_TRAFFIC_BYTES = {"llama8b": 1051010000 + 4268000, "llama8b_k32": 1064188000 + 4393000,
+                     "llama8b_b2k32": 1079315000 + 4162000}
 
 
 def load_peaks():
@@ -346,7 +347,7 @@ def run_stub(args, rank, world, backend):
 SWEEPS = {
     # (head name, V, d, [(B, T, K), ...]): call sizes from 8 paths to the tensor-bound range
     "llama8b": (128256, 4096, [(1, 1, 8), (1, 2, 8), (1, 5, 8), (1, 8, 8), (1, 5, 16), (1, 8, 16), (1, 5, 32),
-                               (1, 8, 32), (3, 5, 20), (4, 8, 16), (8, 8, 16)]),
+                               (1, 7, 32), (1, 8, 32), (3, 5, 20), (4, 8, 16), (8, 8, 16)]),
     "qwen8b": (151936, 4096, [(B, 7, K) for B in (1, 8, 32) for K in (4, 8, 16, 32)]),
     "llama70b": (128256, 8192, [(1, 8, 16), (16, 8, 16)]),
 }
