@@ -1,7 +1,7 @@
 // Fused sm_100a kernel for bf16 heads: Eq. 1 masks (Philox), Eq. 2 masking, Eq. 3 on tcgen05
 // tensor cores with fp32 accumulators in TMEM, and the argmax of Sec. 3.2 in the epilogue.  W is
 // streamed from HBM once per launch and no logit is written (except on request: the debug call
-// and the JS criterion ask for them).  For calls of up to 64 paths or so the masked hidden rows
+// and the JS criterion ask for them).  For calls of up to 48 paths the masked hidden rows
 // exist in shared memory only; for wider calls they are staged once through global memory.
 //
 // Work split.  The vocabulary is cut into one contiguous slice per CTA (one CTA per SM) and
@@ -17,11 +17,17 @@
 //   - one group (the whole slice fits TMEM): builder warps generate the masks with Philox in
 //     registers and write the masked rows of each block into a shared-memory ring, once per call;
 //   - several groups ("staged"): mask_operand_kernel has written the masked rows to a staging
-//     buffer in global memory once per call, and a second TMA ring streams its blocks in.
+//     buffer in global memory once per call.  W tiles and operand blocks share one ring of
+//     "steps": a step is the group's W tiles of one hidden-size block with the operand block
+//     behind them, one barrier for "all of it has landed" and one for "the MMAs are done with
+//     it", so that the issuing warp waits once and commits once per step.  A group takes at most
+//     half of the accumulator slots: the epilogue of one group overlaps the MMAs of the next.
+//     Staged launches run as CTA pairs (see kPair below).
 //
 // Warp roles (14 warps):
 //   warp 0      TMA producer: one thread issues cp.async.bulk.tensor loads of W
-//   warp 1      one thread issues tcgen05.mma and the commits
+//   warp 1      MMA issuer: the whole warp runs the loop converged, one elected lane issues
+//               tcgen05.mma and the commits (their operands then live in uniform registers)
 //   warps 2-5   epilogue: tcgen05.ld the finished accumulators of a group, scale by 1/(1-p),
 //               reduce each column over tiles and lanes to (max, first index), keep the best
 //               per path; warp 2 also allocates and frees TMEM; the last CTA of a one-launch
@@ -800,8 +806,10 @@ struct SmemPlan {
 bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     SmemPlan best{};
     int n_pad = (rows + 15) & ~15;
-    // Staged launches with many operand rows run as CTA pairs: at N >= kPairMinNPad the operand
-    // reads of a lone CTA's MMAs, added to the TMA writes, saturate its shared memory.
+    // Launches of at least DM_STAGED_MIN_NPAD operand rows are staged even where one group would
+    // fit TMEM (two groups: the first epilogue then overlaps the second group's MMAs), and staged
+    // launches of at least kPairMinNPad rows run as CTA pairs: half the MMA issue work and half
+    // the operand bytes per SM.  Measured faster than lone CTAs from 49 paths up.
     const bool force_staged = n_pad >= DM_STAGED_MIN_NPAD && tiles_per_cta > 1;
     best.pair = ((tiles_per_cta > kTmemCols / n_pad || force_staged) && n_pad >= kPairMinNPad) ? 1 : 0;
     if (best.pair) n_pad = (rows + 31) & ~31;
