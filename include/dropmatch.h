@@ -131,11 +131,18 @@ int dropmatch_verify_batched(dm_ctx* ctx, const void* H, const int32_t* draft, i
  * with u[v] = (n + 0.5) / 2^23, n = top 23 bits of word (v mod 4) of
  * Philox4x32-10(counter = (v/4, i + 2^31, t, s mod 2^32), key = seed): the same generator as the
  * masks, on counters the masks never use, so a call is reproducible from (seed, s, t, i) alone.
- * The noise is generated in the epilogue of the head kernel (one Philox call and two logarithms
- * per logit); no logit is written to memory.  Counts, per-position test and scan are unchanged.
- *   temperature > 0;  top_p in (0,1]: the nucleus mass.  top_p < 1 needs all logits of a path at
- *   once (sort and cut) and is not implemented on the device: DM_EUNSUPPORTED.
- * Everything else as for dropmatch_verify_batched. */
+ *   temperature > 0;  top_p in (0,1]: the nucleus mass.
+ * top_p = 1 (temperature sampling): the noise is generated in the epilogue of the head kernel (one
+ * Philox call and two logarithms per logit); no logit is written to memory.
+ * top_p < 1 (nucleus sampling): the nucleus is the tokens in order of decreasing
+ * Softmax(l / temperature) (equal probabilities: increasing id) up to and including the one whose
+ * cumulative probability reaches top_p, and the draw is restricted to it.  The cut needs all logits
+ * of a path at once: the head kernel writes them to the buffer that dm_enable_js reserves (call it
+ * first with room for B*T*K rows, else DM_EWORKSPACE), and a second kernel, one block per path,
+ * finds the boundary by mass (fixed-point sums: the result does not depend on the order of
+ * additions) and draws the token.  Sharded heads (dm_set_vocab_offset) are not supported here: the
+ * nucleus is taken over this context's head.
+ * Counts, per-position test and scan are unchanged; everything else as for dropmatch_verify_batched. */
 int dropmatch_verify_batched_sampled(dm_ctx* ctx, const void* H, const int32_t* draft, int B, int T, int K,
                                      float p, uint64_t seed, uint64_t seq_base, int rule, float temperature,
                                      float top_p, int32_t* out_tokens, int32_t* out_counts,

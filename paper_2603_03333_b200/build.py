@@ -8,7 +8,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libdropmatch.so"
-SOURCES = ["dm_api.cu", "dm_simt.cu", "dm_finalize.cu", "dm_fused_sm100.cu", "dm_noalloc.cu", "dm_js.cu"]
+SOURCES = ["dm_api.cu", "dm_simt.cu", "dm_finalize.cu", "dm_fused_sm100.cu", "dm_noalloc.cu", "dm_js.cu", "dm_sample.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 

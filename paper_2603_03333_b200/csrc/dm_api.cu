@@ -390,11 +390,11 @@ int dropmatch_verify_batched_sampled(dm_ctx* c, const void* H, const int32_t* dr
         return DM_EINVAL;
     if (rule != DM_RULE_NAIVE && rule != DM_RULE_MAJORITY) return DM_EINVAL;
     if (!(temperature > 0.0f) || !(temperature < 1e30f) || !(top_p > 0.0f) || !(top_p <= 1.0f)) return DM_EINVAL;
-    if (top_p < 1.0f) return DM_EUNSUPPORTED;   // the nucleus cut needs every logit of a path at once
     MaskKey mk;
     if (!make_mask_key(p, seed, &mk)) return DM_EINVAL;
-    mk.sample = 1;
     mk.inv_temp = 1.0f / temperature;
+    const int rows = B * T * K;
+    if (top_p < 1.0f && (c->js_logits == nullptr || rows > c->js_max_rows)) return DM_EWORKSPACE;
     DeviceGuard g(c->device);
     if (!g.ok) return DM_ECUDA;
     RowMap map{nullptr, K, T, B, (uint32_t)seq_base, c->mask_mode};
@@ -403,7 +403,35 @@ int dropmatch_verify_batched_sampled(dm_ctx* c, const void* H, const int32_t* dr
     fa.draft = draft; fa.out_hits = out_draft_hits;
     fa.N = 0;
     fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
-    return run_verify(c, H, B * T * K, map, mk, fa, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (top_p >= 1.0f) {   // temperature sampling: Gumbel-max in the epilogue of the head kernel, no logits in memory
+        mk.sample = 1;
+        return run_verify(c, H, rows, map, mk, fa, s);
+    }
+    // Nucleus: the cut needs all logits of a path at once.  The head kernel writes them to the
+    // context's logits buffer (its own argmax is not used), one block per path finds the nucleus
+    // and draws the token, the finalize kernel does the rest.
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    if (rows > c->max_rows) return DM_EWORKSPACE;
+    int impl;
+    st = pick_impl(c, rows, &impl);
+    if (st != DM_OK) return st;
+    int n_slices = 0, launches = 1;
+    if (impl == DM_IMPL_TCGEN05)
+        st = fused_launch(c->fused, c->head, H, B * T, rows, map, mk, &n_slices, c->partials, c->js_logits, c->err, s,
+                          &launches, nullptr, nullptr, nullptr, nullptr, nullptr, c->wait_limit, c->pdl);
+    else
+        st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, c->js_logits, c->err, s);
+    if (st != DM_OK) return st;
+    unsigned long long* packed = c->partials;   // the per-slice partials are not needed: reuse their first row
+    st = launch_nucleus_sample(c->js_logits, c->head.V, rows, map, mk, top_p, c->head.v_offset, packed, s);
+    if (st != DM_OK) return st;
+    fa.err = c->err;
+    st = launch_finalize(packed, 1, rows, fa, s);
+    if (st != DM_OK) return st;
+    c->last_impl = impl;
+    c->last_launches = launches + 2;
+    return DM_OK;
 }
 
 int dropmatch_verify_batched_next(dm_ctx* c, const void* H, const int32_t* draft, int B, int T, int bonus_row,

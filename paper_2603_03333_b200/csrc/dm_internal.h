@@ -98,6 +98,10 @@ int launch_js(const float* logits, const float* draft_prob, float* workspace, si
               int K, const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
               int32_t* out_accept_len, const uint32_t* err, cudaStream_t stream);
 
+// Nucleus sampling on logits [rows][V] in global memory: one packed (key, inverted token id) word per path.
+int launch_nucleus_sample(const float* logits, int V, int rows, const RowMap& map, const MaskKey& mk, float top_p,
+                          int v_offset, unsigned long long* out_packed, cudaStream_t stream);
+
 int launch_debug_masks(int B, int T, int K, int d, const MaskKey& mk, uint32_t seq_base_lo, int shared_masks,
                        uint32_t* out_bits, cudaStream_t stream);
 

@@ -1,7 +1,10 @@
 """GPU parity of the sampling decode rule (dropmatch_verify_batched_sampled) against the oracle:
 the drawn tokens must be identical except where the oracle's two best perturbed keys
 (logit / temperature + Gumbel noise) are closer than the near-tie bound; counts, hits and accepted
-lengths are integer work on the tokens and must match exactly."""
+lengths are integer work on the tokens and must match exactly.  With a nucleus (top_p < 1) the
+GPU sums fp32 probabilities where the oracle sums fp64 ones: where the running mass passes top_p
+within 1e-4 the boundary token may differ, so a token may also equal the oracle's draw at
+top_p * (1 -+ 1e-4); such rows are counted and must stay rare."""
 import numpy as np
 import pytest
 import torch
@@ -57,11 +60,88 @@ def test_cold_temperature_is_the_argmax_call_and_top_p_is_refused():
         plain = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
         for key in ("tokens", "counts", "hits", "accept_len"):
             assert np.array_equal(cold[key], plain[key]), key
-        with pytest.raises(pk.DropMatchError) as e:
+        with pytest.raises(pk.DropMatchError) as e:     # the nucleus needs the logits buffer of dm_enable_js
             ctx.verify_batched_sampled(work.H, work.draft, cfg.K, cfg.p, SEED, temperature=1.0, top_p=0.9)
-        assert e.value.status == binding.EUNSUPPORTED
+        assert e.value.status == binding.EWORKSPACE
         with pytest.raises(pk.DropMatchError) as e:
             ctx.verify_batched_sampled(work.H, work.draft, cfg.K, cfg.p, SEED, temperature=0.0)
         assert e.value.status == binding.EINVAL
+    finally:
+        ctx.close()
+
+
+NUCLEUS_CASES = [
+    (wl.CONFIGS["toy"], 1.0, 0.9),
+    (wl.Config("n_bf16", d=512, V=3000, dtype=wl.BF16, B=2, T=3, K=8, p=0.1), 0.7, 0.5),
+    (wl.Config("n_flat", d=256, V=20000, dtype=wl.BF16, B=1, T=2, K=16, p=0.2), 3.0, 0.95),   # flat: a nucleus of thousands
+    (wl.Config("n_peaked", d=256, V=5000, dtype=wl.BF16, B=2, T=2, K=8, p=0.1), 0.05, 0.3),    # peaked: one or two tokens
+    (wl.Config("n_staged", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1), 1.0, 0.8),   # staged head kernel, 192 paths
+    (wl.Config("n_tiny", d=64, V=37, dtype=wl.BF16, B=1, T=2, K=4, p=0.3), 1.0, 0.6),
+]
+
+
+@pytest.mark.parametrize("cfg,tau,top_p", NUCLEUS_CASES, ids=lambda c: getattr(c, "name", str(c)))
+def test_nucleus_sampling_matches_the_oracle(cfg, tau, top_p):
+    work = wl.make_workload(cfg, device=DEV)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows)
+        ctx.enable_js(cfg.rows, cfg.B * cfg.T)
+        got = to_np(ctx.verify_batched_sampled(work.H, work.draft, cfg.K, cfg.p, SEED, temperature=tau, top_p=top_p,
+                                               seq_base=2))
+        assert ctx.device_error() == 0
+        Wn, Hn, draft = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H), work.draft.cpu().numpy()
+        p32 = float(np.float32(top_p))
+        ref = oracle.verify_batched_sampled(Wn, cfg.dtype, Hn, draft, cfg.K, cfg.p, SEED, temperature=tau, top_p=p32,
+                                            seq_base=2)
+        differ = got["tokens"] != ref["tokens"]
+        boundary_cases = 0
+        for b, t, i in np.argwhere(differ & (ref["gap"] >= 2e-2)):
+            logits = oracle.logits_row(Wn, cfg.dtype, Hn[b, t], cfg.p, SEED, 2 + b, t, i)
+            alts = {oracle.sample_row(logits, tau, p32 * f, SEED, 2 + b, t, i)[0] for f in (1 - 1e-4, 1 + 1e-4)}
+            assert got["tokens"][b, t, i] in alts, (b, t, i)
+            boundary_cases += 1
+        assert boundary_cases <= max(1, cfg.rows // 50)
+        # every drawn token lies in the oracle's nucleus at a slightly larger mass
+        for b in range(cfg.B):
+            for t in range(cfg.T):
+                for i in range(0, cfg.K, max(1, cfg.K // 2)):
+                    logits = oracle.logits_row(Wn, cfg.dtype, Hn[b, t], cfg.p, SEED, 2 + b, t, i)
+                    assert oracle.nucleus(logits, tau, min(1.0, p32 * (1 + 1e-3)))[got["tokens"][b, t, i]]
+                cnt, hits = oracle.counts(got["tokens"][b, t], int(draft[b, t]))
+                assert np.array_equal(got["counts"][b, t], cnt) and got["hits"][b, t] == hits
+            assert got["accept_len"][b] == oracle.accept_chain(got["tokens"][b], draft[b])
+        again = to_np(ctx.verify_batched_sampled(work.H, work.draft, cfg.K, cfg.p, SEED, temperature=tau, top_p=top_p,
+                                                 seq_base=2))
+        assert np.array_equal(again["tokens"], got["tokens"])       # reproducible bit for bit
+    finally:
+        ctx.close()
+
+
+@pytest.mark.parametrize("top_p", [1.0, 0.9])
+def test_sampling_on_the_llama8b_head(top_p):
+    """Full-size head (V=128256, d=4096), 16 paths: temperature sampling in the fused epilogue and
+    nucleus sampling through the logits buffer, each against the oracle."""
+    cfg = wl.CONFIGS["llama8b"].with_(T=2)
+    work = wl.make_workload(cfg, device=DEV)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=cfg.rows)
+        if top_p < 1.0:
+            ctx.enable_js(cfg.rows, cfg.B * cfg.T)
+        got = to_np(ctx.verify_batched_sampled(work.H, work.draft, cfg.K, cfg.p, SEED, temperature=0.8, top_p=top_p))
+        assert ctx.device_error() == 0 and ctx.last_impl() == binding.IMPL_TCGEN05
+        Wn, Hn, draft = wl.to_numpy_storage(work.W), wl.to_numpy_storage(work.H), work.draft.cpu().numpy()
+        p32 = float(np.float32(top_p))
+        ref = oracle.verify_batched_sampled(Wn, cfg.dtype, Hn, draft, cfg.K, cfg.p, SEED, temperature=0.8, top_p=p32)
+        for b, t, i in np.argwhere((got["tokens"] != ref["tokens"]) & (ref["gap"] >= 2e-2)):
+            assert top_p < 1.0
+            logits = oracle.logits_row(Wn, cfg.dtype, Hn[b, t], cfg.p, SEED, b, t, i)
+            alts = {oracle.sample_row(logits, 0.8, p32 * f, SEED, b, t, i)[0] for f in (1 - 1e-4, 1 + 1e-4)}
+            assert got["tokens"][b, t, i] in alts
+        for t in range(cfg.T):
+            cnt, hits = oracle.counts(got["tokens"][0, t], int(draft[0, t]))
+            assert np.array_equal(got["counts"][0, t], cnt) and got["hits"][0, t] == hits
+        assert got["accept_len"][0] == oracle.accept_chain(got["tokens"][0], draft[0])
     finally:
         ctx.close()
