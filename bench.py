@@ -2,8 +2,9 @@
 """Benchmark of the DropMatch verification path: verify calls/s on the Llama-3-8B-shaped head.
 
 One step = one whole verify call (Eq. 1 masks, Eq. 2-3 masked head, per-path argmax, token
-counts, acceptance scan: one launch of the fused kernel at this size) on one batch of synthetic
-input: d=4096, V=128256, bf16, T=5 draft positions, K=8 dropout paths, p=0.1, B=1.
+counts, acceptance scan: at this size a 2 us mask pass and one launch of the fused kernel, whose
+last CTA finishes the call) on one batch of synthetic input: d=4096, V=128256, bf16, T=5 draft
+positions, K=8 dropout paths, p=0.1, B=1.
 Prints ONE JSON line (rank 0).  `--gpus N` run as plain `python bench.py` starts N ranks itself
 (one per GPU, independent replicas); under torchrun it joins the ranks it is given.
 `--impl reference` times the CPU oracle instead.
@@ -30,7 +31,7 @@ WORKLOAD = "llama8b"   # Llama-3-8B-shaped head: the configuration the metric is
 
 # DRAM bytes (read + write) of one fused head-kernel launch on this workload, from the ncu capture
 # summarised in profiles/; None until a capture exists.
-NCU_TRAFFIC_BYTES = {"llama8b": 1051010000 + 4268000, "llama8b_k32": 1064188000 + 4393000,
+NCU_TRAFFIC_BYTES = {"llama8b": 1051650000 + 4317000, "llama8b_k32": 1064188000 + 4393000,
                      "llama8b_b2k32": 1079315000 + 4162000}
 
 

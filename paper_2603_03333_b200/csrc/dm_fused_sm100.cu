@@ -1,7 +1,7 @@
 // Fused sm_100a kernel for bf16 heads: Eq. 1 masks (Philox), Eq. 2 masking, Eq. 3 on tcgen05
 // tensor cores with fp32 accumulators in TMEM, and the argmax of Sec. 3.2 in the epilogue.  W is
 // streamed from HBM once per launch and no logit is written (except on request: the debug call
-// and the JS criterion ask for them).  For calls of up to 48 paths the masked hidden rows
+// and the JS criterion ask for them).  For calls of up to 32 paths the masked hidden rows
 // exist in shared memory only; for wider calls they are staged once through global memory.
 //
 // Work split.  The vocabulary is cut into one contiguous slice per CTA (one CTA per SM) and
@@ -61,10 +61,10 @@ constexpr int kIdlePollNs = 500;            // ... and of one that completes onc
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort flag
 #ifndef DM_PAIR_MIN_NPAD
-#define DM_PAIR_MIN_NPAD 64
+#define DM_PAIR_MIN_NPAD 48
 #endif
 #ifndef DM_STAGED_MIN_NPAD
-#define DM_STAGED_MIN_NPAD 64   // launches at least this wide are staged even if the slice would fit TMEM as one group
+#define DM_STAGED_MIN_NPAD 48   // launches at least this wide are staged even if the slice would fit TMEM as one group
 #endif
 constexpr int kPairMinNPad = DM_PAIR_MIN_NPAD;   // staged launches at least this wide run as CTA pairs
 
@@ -166,7 +166,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             ptx::mbar_init(b_ready + 8 * s, P.staged ? 1 : wps);
             ptx::mbar_init(b_empty + 8 * s, 1);
         }
-        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, kPair ? 16 : P.staged ? 8 : 4); }
+        for (int s = 0; s < P.n_slots; ++s) { ptx::mbar_init(slot_full + 8 * s, 1); ptx::mbar_init(slot_empty + 8 * s, kPair ? 16 : P.staged ? 8 : 12); }
         ptx::mbar_init(dealloc_bar, 1);
         *s_abort = 0;
         *s_never = 0;
@@ -507,7 +507,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(b_ready + 8 * grp);
         }
-        return;
+        // The operand is built (once per call): these warps now help with the epilogue as two more sets.
     }
 
     {
@@ -516,8 +516,8 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // lanes 32*(w mod 4)..+31; the warps of a lane quarter share the column chunks.
         if (P.pdl) ptx::griddep_wait();       // global writes (and the shared per-row best) only after the kernel ahead
         const int ew = warp & 3;                      // lane quarter = row of s_best
-        const int set = warp < kFirstExpWarp ? 0 : 1;
-        const int n_sets = P.staged ? 2 : 1;
+        const int set = warp < kFirstExpWarp ? 0 : 1 + (warp - kFirstExpWarp) / 4;
+        const int n_sets = P.staged ? 2 : 3;
         const int lane_base = ew * 32;                // TMEM lanes this warp may read
         // A group's accumulators finish together.  Columns are then taken 16 at a time and, for
         // each, the group's tiles are walked with a per-lane running maximum (a lane always sees
@@ -809,7 +809,9 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     // Launches of at least DM_STAGED_MIN_NPAD operand rows are staged even where one group would
     // fit TMEM (two groups: the first epilogue then overlaps the second group's MMAs), and staged
     // launches of at least kPairMinNPad rows run as CTA pairs: half the MMA issue work and half
-    // the operand bytes per SM.  Measured faster than lone CTAs from 49 paths up.
+    // the operand bytes per SM.  Measured faster than lone CTAs, and than the one-group mode with
+    // its in-kernel Philox builders, from 33 paths up (equal on boxes that hold their clock, 4-25 us
+    // faster on boxes that the power cap slows down).
     const bool force_staged = n_pad >= DM_STAGED_MIN_NPAD && tiles_per_cta > 1;
     best.pair = ((tiles_per_cta > kTmemCols / n_pad || force_staged) && n_pad >= kPairMinNPad) ? 1 : 0;
     if (best.pair) n_pad = (rows + 31) & ~31;

@@ -60,13 +60,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
-// The same wait for a whole warp: lane 0 polls, the other lanes pick the outcome up.
+// The same wait for a whole warp: lane 0 polls, the other lanes pick the outcome up.  Every lane
+// runs the loop, and every branch in it depends on a warp-wide value only, so that the warp
+// leaves it converged: were lane 0 to spin on its own, the code behind the wait could run
+// once for lane 0 and once more for the other lanes.
 template <int SLEEP_NS>
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                long long limit_cycles) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait<SLEEP_NS>(bar, parity, abort_flag, limit_cycles) ? 1 : 0;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+    const bool poller = (threadIdx.x & 31) == 0;
+    long long t0 = 0;
+    for (int tries = 0;; ++tries) {
+        int state = 0;   // 1: phase complete, 2: give up
+        if (poller) {
+            if (mbar_try_wait(bar, parity)) state = 1;
+            else if (*abort_flag) state = 2;
+            else if (tries == 1) t0 = clock64();
+            else if (tries > 1 && clock64() - t0 > limit_cycles) { *abort_flag = 1; state = 2; }
+        }
+        state = __shfl_sync(0xFFFFFFFFu, state, 0);
+        if (state != 0) return state == 1;
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+    }
 }
 
 // The same wait for a warp that must stay converged: every lane runs the loop and every branch

@@ -56,15 +56,16 @@ def _check_masks(ctx, cfg, paths, seq_base=0):
 
 
 def test_bench_workload_every_path():
-    """The call bench.py times (Llama-3-8B head, B=1, T=5, K=8: 40 paths, one launch) against the
-    oracle's whole call: all 40 tokens, counts, hits and the accepted length."""
+    """The call bench.py times (Llama-3-8B head, B=1, T=5, K=8: 40 paths; the mask pass and the head
+    kernel, which finishes the call itself) against the oracle's whole call: all 40 tokens, counts,
+    hits and the accepted length."""
     cfg = wl.CONFIGS["llama8b"]
     work = wl.make_workload(cfg, device=DEV)
     ctx = pk.Context(0)
     try:
         ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
         got = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED))
-        assert ctx.device_error() == 0 and ctx.last_impl() == binding.IMPL_TCGEN05 and ctx.last_launches() == 1
+        assert ctx.device_error() == 0 and ctx.last_impl() == binding.IMPL_TCGEN05 and ctx.last_launches() == 2
         draft = work.draft.cpu().numpy()
         ref = oracle.verify_batched(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H), draft,
                                     cfg.K, cfg.p, SEED)
