@@ -168,10 +168,14 @@ int dropmatch_verify_batched_next(dm_ctx* ctx, const void* H, const int32_t* dra
 
 /* Same as dropmatch_verify_batched, but H, draft and all outputs are HOST pointers (pinned or
  * pageable).  Pinned buffers (cudaHostAlloc, cudaHostRegister, torch pin_memory) are used where
- * they are: a small kernel fetches the inputs over the host link while the head kernel already
- * streams W, and the results are written by the device straight into the caller's arrays.
- * Pageable buffers go through the context's own pinned buffers (one memcpy each way).  The call
- * returns after `stream` has drained, with the results in place.  Whether a pointer is pinned is
+ * they are: the first kernel of the call (the mask pass, or a small copy kernel) fetches the
+ * inputs over the host link while the head kernel already streams W, and the results are
+ * written by the device straight into the caller's arrays.  Pageable buffers go through the
+ * context's own pinned buffers (one memcpy each way).  The call returns once every result is in
+ * place: the block that finishes the call writes a word into host memory behind its results and
+ * the host waits for that word (or, where several blocks finish the call, for `stream` to
+ * drain), so the call's last kernel may still be retiring on `stream` for a few microseconds
+ * after the return; work queued on `stream` afterwards is ordered behind it as usual.  Whether a pointer is pinned is
  * looked up once and remembered (the last eight pointers): do not unpin or free a buffer and
  * reuse its address as pageable memory without a dm_set_head in between.  Needs
  * B*T <= max_hidden_rows of dm_set_head; H_host 16-byte aligned.  out_draft_hits may be NULL. */

@@ -97,7 +97,15 @@ def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream(device) -> ctypes.c_void_p:
+    # the handle of torch's current stream on `device` (the short way where this torch has it)
+    if _raw_stream is not None:
+        index = device if isinstance(device, int) else torch.device(device).index
+        if index is not None:
+            return ctypes.c_void_p(_raw_stream(index))
     return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
 
 

@@ -1,6 +1,7 @@
 // C ABI of libdropmatch: argument checks, workspace, kernel choice.  See include/dropmatch.h.
 #include <math.h>
 #include <string.h>
+#include <atomic>
 #include <new>
 #include <vector>
 
@@ -29,6 +30,10 @@ struct dm_ctx {
     unsigned char* pin_in_dev = nullptr;     // the same memory as the device sees it
     int32_t* pin_out = nullptr;              // pinned host, mapped
     int32_t* pin_out_dev = nullptr;          // the same memory as the device sees it
+    size_t done_off = 0;                     // the "results written" word of host-buffer calls: pin_out[done_off]
+    uint32_t done_seq = 0;                   // its value for the latest host-buffer call
+    const HostInputs* host_in = nullptr;     // set while a host-buffer call is being launched
+    bool done_armed = false;                 // did the latest launch hand the word to a single finishing block?
     size_t ws_bytes = 0;
     // host pointers the host-buffer entry point has already looked up: device alias, or null if pageable
     struct HostAlias { const void* host = nullptr; void* dev = nullptr; };
@@ -122,6 +127,11 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
                const FinalizeArgs& fa_in, cudaStream_t stream, float* logits_out = nullptr) {
     FinalizeArgs fa = fa_in;
     fa.err = c->err;   // results are replaced by "nothing accepted" if a kernel of the call gives up on a wait
+    const HostInputs* host = c->host_in;
+    if (host != nullptr) {
+        fa.done = reinterpret_cast<uint32_t*>(c->pin_out_dev + c->done_off);
+        fa.done_value = c->done_seq;
+    }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
     if (rows > c->max_rows) return DM_EWORKSPACE;
     if (finalize_smem_bytes(fa.T, fa.K + fa.plain, fa.N) > 200 * 1024) return DM_EUNSUPPORTED;
@@ -144,10 +154,17 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
                           logits_out, c->err, stream, &launches, &fa, c->err + 1,
-                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded, nullptr, c->wait_limit, c->pdl);
+                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded, nullptr, c->wait_limit, c->pdl, host);
     else {
+        if (host != nullptr) {
+            st = launch_host_gather(host->h_src, host->h_bytes, host->draft_src, host->n_draft, host->h_dst,
+                                    host->draft_dst, stream);
+            if (st != DM_OK) return st;
+            H = host->h_dst;
+            ++launches;
+        }
         st = launch_simt(c->head, H, rows, map, mk, &n_slices, c->partials, logits_out, c->err, stream);
-        launches = 1;
+        ++launches;
     }
     if (ev_end != nullptr) {
         cudaEventRecord(ev_end, stream);
@@ -159,6 +176,7 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
         if (st != DM_OK) return st;
         ++launches;
     }
+    c->done_armed = host != nullptr && (folded || fa.B == 1);   // one block finishes the call and writes the word
     c->last_impl = impl;
     c->last_launches = launches;
     return DM_OK;
@@ -233,7 +251,8 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
     // that the fused kernel's CTAs reduce into when one launch covers the call (zero between calls)
     const size_t n_part = ((size_t)kMaxSlices + 1) * max_rows * sizeof(unsigned long long);
     const size_t n_in = (size_t)max_hidden_rows * d * elem + 16 + (size_t)max_hidden_rows * sizeof(int32_t);
-    const size_t n_out = ((size_t)2 * max_hidden_rows + 2 * (size_t)max_rows) * sizeof(int32_t);
+    c->done_off = (((size_t)2 * max_hidden_rows + 2 * (size_t)max_rows) + 15) & ~static_cast<size_t>(15);
+    const size_t n_out = (c->done_off + 16) * sizeof(int32_t);
     void* out_dev = nullptr;
     void* in_dev = nullptr;
     if (cudaMalloc(&c->partials, n_part) != cudaSuccess || cudaMalloc(&c->stage_in, n_in) != cudaSuccess ||
@@ -248,6 +267,8 @@ int dm_set_head(dm_ctx* c, const void* W, int V, int d, int dtype, int max_rows,
         return DM_ECUDA;
     }
     c->pin_out_dev = static_cast<int32_t*>(out_dev);
+    c->pin_out[c->done_off] = 0;
+    c->done_seq = 0;
     c->pin_in_dev = static_cast<unsigned char*>(in_dev);
     for (dm_ctx::HostAlias& a : c->aliases) a = dm_ctx::HostAlias{};
     c->ws_bytes = n_part + n_in;
@@ -503,8 +524,7 @@ int dropmatch_verify_batched_host(dm_ctx* c, const void* H_host, const int32_t* 
         d_src = c->pin_in_dev + draft_off;
     }
     int32_t* draft_dev = reinterpret_cast<int32_t*>(c->stage_in + draft_off);
-    st = launch_host_gather(h_src, h_bytes, static_cast<const int32_t*>(d_src), (int)hidden, c->stage_in, draft_dev, s);
-    if (st != DM_OK) return st;
+    const HostInputs host{h_src, h_bytes, static_cast<const int32_t*>(d_src), (int)hidden, c->stage_in, draft_dev};
     // Outputs.  The kernels write them into host memory the device can reach (a few hundred bytes
     // crossing to the host), so that no device-to-host copy is queued behind the call: straight into
     // the caller's arrays if those are pinned, else into the context's mapped buffer.
@@ -513,11 +533,34 @@ int dropmatch_verify_batched_host(dm_ctx* c, const void* H_host, const int32_t* 
     int32_t* o_len = static_cast<int32_t*>(device_alias(c, out_accept_len_host));
     int32_t* o_hits = out_draft_hits_host ? static_cast<int32_t*>(device_alias(c, out_draft_hits_host)) : nullptr;
     int32_t* d_out = c->pin_out_dev;
+    c->host_in = &host;   // the first kernel of the call fetches the inputs
+    ++c->done_seq;
+    c->done_armed = false;
     st = dropmatch_verify_batched(c, c->stage_in, draft_dev, B, T, K, p, seed, seq_base, rule,
                                   o_tok ? o_tok : d_out, o_cnt ? o_cnt : d_out + rows,
                                   o_hits ? o_hits : d_out + 2 * rows, o_len ? o_len : d_out + 2 * rows + hidden, stream);
+    c->host_in = nullptr;
     if (st != DM_OK) return st;
-    if (cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    // The block that finishes the call writes a word into host memory behind the results: poll it
+    // rather than wait for the stream to report the kernel retired.  The stream is asked now and
+    // then all the same, so that a launch that failed, or a call whose end no single block sees,
+    // ends the loop too.
+    bool seen = false;
+    if (c->done_armed) {
+        const volatile uint32_t* word = reinterpret_cast<const volatile uint32_t*>(c->pin_out + c->done_off);
+        for (unsigned spins = 1;; ++spins) {
+            if (*word == c->done_seq) { seen = true; break; }
+            if ((spins & 2047u) == 0) {
+                if (cudaStreamQuery(s) != cudaErrorNotReady) break;
+                cudaGetLastError();   // "not ready" is no error: do not leave it for the next call to find
+            }
+#if defined(__x86_64__)
+            __builtin_ia32_pause();
+#endif
+        }
+        std::atomic_thread_fence(std::memory_order_acquire);
+    }
+    if (!seen && cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
     if (!o_tok) memcpy(out_tokens_host, c->pin_out, (size_t)rows * sizeof(int32_t));
     if (!o_cnt) memcpy(out_counts_host, c->pin_out + rows, (size_t)rows * sizeof(int32_t));
     if (!o_len) memcpy(out_accept_len_host, c->pin_out + 2 * rows + hidden, (size_t)B * sizeof(int32_t));

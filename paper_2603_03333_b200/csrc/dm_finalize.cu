@@ -9,6 +9,11 @@ __global__ void __launch_bounds__(256)
 finalize_kernel(const unsigned long long* __restrict__ partials, int n_slices, int rows, FinalizeArgs a) {
     extern __shared__ int32_t sm[];
     finalize_sequence(partials, n_slices, rows, a, (int)blockIdx.x, sm, (int)threadIdx.x, (int)blockDim.x, BlockSync{});
+    if (a.done != nullptr && gridDim.x == 1) {   // one block wrote every result: tell the waiting host
+        __threadfence_system();
+        __syncthreads();
+        if (threadIdx.x == 0) *reinterpret_cast<volatile uint32_t*>(a.done) = a.done_value;
+    }
 }
 
 // One packed word per row: the maximum over the slices (argmax with the smallest index on ties).

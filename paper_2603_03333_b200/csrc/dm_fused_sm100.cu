@@ -714,6 +714,11 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                                               WarpSync{});
                     ptx::bar_sync(1, 4 * 32);
                 }
+                if (P.fin.done != nullptr) {   // a host-buffer call: every result is written, tell the waiting host
+                    __threadfence_system();
+                    ptx::bar_sync(1, 4 * 32);
+                    if (tid_e == 0) *reinterpret_cast<volatile uint32_t*>(P.fin.done) = P.fin.done_value;
+                }
                 for (int n = tid_e; n < P.rows_total; n += 4 * 32) P.best[n] = 0ull;   // ready for the next call
                 if (tid_e == 0) *P.ticket = 0u;
             }
@@ -729,8 +734,11 @@ __global__ void __launch_bounds__(256)
 mask_operand_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat16* __restrict__ out, int rows, int d,
                     RowMap map, uint32_t key0, uint32_t key1, uint32_t thr, uint32_t* __restrict__ err) {
     // The head kernel behind this one may be scheduled at once: it streams W until its operand
-    // producer needs these rows, and that thread waits for this kernel to finish.
+    // producer needs these rows, and that thread waits for this kernel to finish.  This kernel may
+    // itself have been scheduled early: the kernel ahead may still read the staging buffer or
+    // write H, so nothing is touched before it has finished.
     ptx::griddep_launch_dependents();
+    ptx::griddep_wait();
     const int chunks = d >> 3;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)rows * chunks) return;
@@ -746,6 +754,42 @@ mask_operand_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat16* __restri
     o.z = hv.z & mask_pair(mbits >> 4);
     o.w = hv.w & mask_pair(mbits >> 6);
     *reinterpret_cast<uint4*>(out + (size_t)r * d + c * 8) = o;
+}
+
+// The same for the regular row order (paths of a position next to each other): a block takes 32
+// chunks of one hidden row, fetches them once and writes them under the mask of every path of the
+// row, eight paths at a time.  H may then be host memory that the device can read (the host-buffer
+// call): each hidden element crosses the host link once; the draft tokens of such a call ride along.
+__global__ void __launch_bounds__(256)
+mask_operand_by_position_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat16* __restrict__ out, int d,
+                                RowMap map, uint32_t key0, uint32_t key1, uint32_t thr,
+                                const int32_t* __restrict__ draft_src, int32_t* __restrict__ draft_dst, int n_draft) {
+    ptx::griddep_launch_dependents();
+    ptx::griddep_wait();   // (see mask_operand_kernel)
+    __shared__ uint4 s_h[32];
+    const int chunks = d >> 3, tiles = (chunks + 31) >> 5;
+    const int q = (int)(blockIdx.x / tiles), c = (int)(blockIdx.x % tiles) * 32 + (threadIdx.x & 31);
+    const int pl = threadIdx.x >> 5;
+    if (draft_src != nullptr && blockIdx.x == 0)
+        for (int x = threadIdx.x; x < n_draft; x += 256) draft_dst[x] = draft_src[x];
+    if (pl == 0 && c < chunks) s_h[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(H + (size_t)q * d + c * 8));
+    __syncthreads();
+    if (c >= chunks) return;
+    const uint4 hv = s_h[threadIdx.x & 31];
+    const int kp = map.K + map.plain_extra;
+    for (int i = pl; i < kp; i += 8) {
+        const int r = q * kp + i;
+        RowKey k;
+        row_key(map, r, k);   // always valid in the regular order
+        const uint32_t mbits = keep4((uint32_t)(2 * c), k, key0, key1, thr) |
+                               (keep4((uint32_t)(2 * c + 1), k, key0, key1, thr) << 4);
+        uint4 o;
+        o.x = hv.x & mask_pair(mbits);
+        o.y = hv.y & mask_pair(mbits >> 2);
+        o.z = hv.z & mask_pair(mbits >> 4);
+        o.w = hv.w & mask_pair(mbits >> 6);
+        *reinterpret_cast<uint4*>(out + (size_t)r * d + c * 8) = o;
+    }
 }
 
 }  // namespace
@@ -948,14 +992,48 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
     return DM_OK;
 }
 
+namespace {
+
+// The mask pass over all rows of a call: by position in the regular row order (H is then read once
+// per element, and the drafts of a host-buffer call may ride along), by row for explicit row lists.
+int launch_mask_operand(int d, const void* H, int rows, const RowMap& map, const MaskKey& mk, __nv_bfloat16* out,
+                        uint32_t* err, cudaStream_t stream, bool pdl, const int32_t* draft_src = nullptr,
+                        int32_t* draft_dst = nullptr, int n_draft = 0) {
+    // With programmatic stream serialization the pass is scheduled while the kernel ahead (the head
+    // kernel of the previous call, say) drains, and so is the head kernel behind it: its prologue
+    // and the fill of its W ring then overlap that tail.  Not for explicit row lists, which could
+    // themselves be the output of the kernel ahead.
+    cudaLaunchConfig_t cfg{};
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = (pdl && map.sel == nullptr) ? 1 : 0;
+    const __nv_bfloat16* Hb = static_cast<const __nv_bfloat16*>(H);
+    cudaError_t e;
+    if (map.sel == nullptr) {
+        const int kp = map.K + map.plain_extra, tiles = (d / 8 + 31) / 32;
+        if (rows % kp != 0) return DM_EINVAL;
+        cfg.gridDim = dim3((unsigned)((rows / kp) * tiles));
+        e = cudaLaunchKernelEx(&cfg, mask_operand_by_position_kernel, Hb, out, d, map, mk.key0, mk.key1, mk.thr,
+                               draft_src, draft_dst, n_draft);
+    } else {
+        const long long n_threads = (long long)rows * (d / 8);
+        cfg.gridDim = dim3((unsigned)((n_threads + 255) / 256));
+        e = cudaLaunchKernelEx(&cfg, mask_operand_kernel, Hb, out, rows, d, map, mk.key0, mk.key1, mk.thr, err);
+    }
+    if (e != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+}
+
+}  // namespace
+
 int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
                         void* out, uint32_t* err, cudaStream_t stream) {
     if (head.dtype != DM_BF16 || head.d % 8 != 0) return DM_EUNSUPPORTED;
-    const long long n_threads = (long long)rows * (head.d / 8);
-    mask_operand_kernel<<<(unsigned)((n_threads + 255) / 256), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(H), static_cast<__nv_bfloat16*>(out), rows, head.d, map, mk.key0, mk.key1,
-        mk.thr, err);
-    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
+    return launch_mask_operand(head.d, H, rows, map, mk, static_cast<__nv_bfloat16*>(out), err, stream, false);
 }
 
 void fused_destroy(FusedState* fs) {
@@ -968,16 +1046,13 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out,
-                 unsigned long long* packed_out, long long wait_limit, bool allow_pdl) {
+                 unsigned long long* packed_out, long long wait_limit, bool allow_pdl, const HostInputs* host) {
     if (folded_out) *folded_out = false;
     if (fs == nullptr || !fused_supported(head, rows) || fs->geo[0].n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
     // Slices of one-block launches: an even count (pairs need one); a CTA whose slice lies past the
     // end of W contributes empty partials.
     const int slices1 = (fs->geo[0].n_ctas + 1) & ~1;
     const int slices2 = (fs->geo[1].n_ctas + 1) & ~1;
-    // Two full blocks of 256 paths are taken together when the launch is tensor-bound anyway: the
-    // two CTAs that share a vocabulary slice stream the same W tiles side by side, so that W comes
-    // from HBM once per 512 paths (the second reader hits L2) and a CTA runs twice as many tiles.
     // More than 256 paths left: two row blocks (of 256, or of half the rest) are taken in one
     // launch.  The two CTAs that share a vocabulary slice stream the same W tiles side by side, so
     // W comes from HBM once for both blocks (the second reader hits L2) and a CTA runs twice as
@@ -992,6 +1067,27 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
     }
     int launches = 0;
     bool operand_staged = false;
+    if (host != nullptr) {
+        // Inputs of the host-buffer call.  If the call's masked rows are staged in the regular row
+        // order, the mask pass reads H where it is and brings the drafts along; otherwise a small
+        // kernel copies both into the device staging buffer first.
+        SmemPlan first;
+        const int first_rows = rows < kMaxNPad ? rows : kMaxNPad;
+        const bool direct = map.sel == nullptr && fs->staging != nullptr && rows <= fs->staging_rows &&
+                            plan_smem(first_rows, fs->geo[0].tiles_per_cta, &first) && first.staged;
+        if (direct) {
+            const int st = launch_mask_operand(head.d, host->h_src, rows, map, mk, fs->staging, err, stream, allow_pdl,
+                                               host->draft_src, host->draft_dst, host->n_draft);
+            if (st != DM_OK) return st;
+            operand_staged = true;
+        } else {
+            const int st = launch_host_gather(host->h_src, host->h_bytes, host->draft_src, host->n_draft, host->h_dst,
+                                              host->draft_dst, stream);
+            if (st != DM_OK) return st;
+        }
+        H = host->h_dst;   // (never read when the operand is staged)
+        ++launches;
+    }
     for (int row0 = 0; row0 < rows;) {
         const int left = rows - row0;
         int row_blocks = 1, block_rows = left < kMaxNPad ? left : kMaxNPad;
@@ -1022,10 +1118,8 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         if (plan.staged && !operand_staged) {
             // one pass over all rows of the call; the launches below read their own rows of it
             if (fs->staging == nullptr || rows > fs->staging_rows) return DM_EWORKSPACE;
-            const long long n_threads = (long long)rows * (head.d / 8);
-            mask_operand_kernel<<<(unsigned)((n_threads + 255) / 256), 256, 0, stream>>>(
-                static_cast<const __nv_bfloat16*>(H), fs->staging, rows, head.d, map, mk.key0, mk.key1, mk.thr, err);
-            if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
+            const int st = launch_mask_operand(head.d, H, rows, map, mk, fs->staging, err, stream, allow_pdl);
+            if (st != DM_OK) return st;
             operand_staged = true;
             ++launches;
         }

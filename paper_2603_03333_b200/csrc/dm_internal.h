@@ -53,6 +53,10 @@ struct FinalizeArgs {
     // device error word of the call's context (or null): if it is set when the results are about to
     // be written, a kernel of the call gave up on a wait and the partial maxima mean nothing
     const uint32_t* err;
+    // Host-buffer calls: a word in host memory that receives `done_value` once every result of the
+    // call has been written (only when one block finishes the whole call), or null.
+    uint32_t* done;
+    uint32_t done_value;
 };
 
 // Reduce the per-slice partial argmaxes to one packed word per row (no histogram, no acceptance).
@@ -73,12 +77,24 @@ struct FusedState;
 bool fused_supported(const HeadDesc& head, int rows);
 int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int max_hidden_rows, size_t* bytes);
 void fused_destroy(FusedState* fs);
+// Inputs of a host-buffer call: where the device can read them (pinned host memory) and where
+// the kernels of the call expect them (device staging).
+struct HostInputs {
+    const void* h_src;
+    size_t h_bytes;
+    const int32_t* draft_src;
+    int n_draft;
+    void* h_dst;
+    int32_t* draft_dst;
+};
+
 int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidden, int rows,
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
                  unsigned long long* best = nullptr, bool* folded_out = nullptr,
-                 unsigned long long* packed_out = nullptr, long long wait_limit = 0, bool allow_pdl = true);
+                 unsigned long long* packed_out = nullptr, long long wait_limit = 0, bool allow_pdl = true,
+                 const HostInputs* host = nullptr);
 
 // The staged masked operand of the tensor-core kernel (Eq. 1 and the numerator of Eq. 2), written to `out`.
 int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
