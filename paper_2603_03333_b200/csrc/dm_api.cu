@@ -620,11 +620,12 @@ int dropmatch_verify_js(dm_ctx* c, const void* H, const int32_t* draft, const fl
     fa.out_tokens = out_tokens; fa.out_counts = out_counts; fa.out_accept_len = out_accept_len;
     st = run_verify(c, H, (int)rows, map, mk, fa, s, c->js_logits);
     if (st != DM_OK) return st;
-    st = launch_js(c->js_logits, draft_prob, c->js_ws,
-                   js_workspace_floats(c->head.V, c->js_max_rows, c->js_max_hidden) - 4, c->head.V, B, T, K, out_tokens,
-                   draft, out_js, out_js_ok, out_accept_len, c->err, s);
+    int js_launches = 0;
+    st = launch_js(c->js_logits, draft_prob, c->js_ws, js_words_offset(c->head.V, c->js_max_rows, c->js_max_hidden),
+                   c->js_max_hidden, c->head.V, B, T, K, out_tokens, draft, out_js, out_js_ok, out_accept_len, c->err, c->wait_limit, s,
+                   &js_launches);
     if (st != DM_OK) return st;
-    c->last_launches += K <= 32 ? 2 : 3;
+    c->last_launches += js_launches;
     return DM_OK;
 }
 

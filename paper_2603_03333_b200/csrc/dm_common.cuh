@@ -14,7 +14,8 @@ enum : uint32_t {
     ERR_WAIT_OPERAND = 3,   // MMA issuer gave up waiting for the masked operand
     ERR_WAIT_ACC_FULL = 4,  // epilogue gave up waiting for an accumulator
     ERR_WAIT_ACC_EMPTY = 5, // MMA issuer gave up waiting for a drained accumulator
-    ERR_BAD_ROW = 6         // debug row selection out of range
+    ERR_BAD_ROW = 6,        // debug row selection out of range
+    ERR_WAIT_JS = 7         // a block of the one-kernel JS sweep gave up waiting for the other blocks of its position
 };
 
 // One path ("row") of a call: which hidden row it masks and its mask key words.

@@ -108,11 +108,12 @@ int launch_read_stream(const void* ptr, size_t bytes, unsigned int* sink, int sm
 
 // JS-divergence acceptance (Eq. 4, Eq. 5, Algorithm 1) on logits [B*T*K][V] written by a head kernel.
 int js_chunks(int V, int n_pos);
-size_t js_workspace_floats(int V, int max_rows, int max_hidden);   // the last four floats hold the ticket word (zero)
+size_t js_workspace_floats(int V, int max_rows, int max_hidden);
+size_t js_words_offset(int V, int max_rows, int max_hidden);       // where the ticket and counter words start (zero between calls)
 constexpr int kJsMaxPositions = 65535;   // B*T of one JS call (a grid dimension)
-int launch_js(const float* logits, const float* draft_prob, float* workspace, size_t ticket_offset, int V, int B, int T,
+int launch_js(const float* logits, const float* draft_prob, float* workspace, size_t words_offset, int max_hidden, int V, int B, int T,
               int K, const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
-              int32_t* out_accept_len, const uint32_t* err, cudaStream_t stream);
+              int32_t* out_accept_len, uint32_t* err, long long wait_limit, cudaStream_t stream, int* launches_out);
 
 // Nucleus sampling on logits [rows][V] in global memory: one packed (key, inverted token id) word per path.
 int launch_nucleus_sample(const float* logits, int V, int rows, const RowMap& map, const MaskKey& mk, float top_p,

@@ -18,6 +18,11 @@ pytestmark = pytest.mark.gpu
 SEED = wl.MASK_SEED
 DEV = "cuda:0"
 JS_ABS, JS_REL = 2e-5, 2e-3
+LAUNCHES = {}     # kernels of the latest verify_js call of each configuration
+# head kernel(s) (+ the mask pass of staged operands) + the sweeps: one cooperative kernel where the
+# call's logits fit the shared memory of the GPU, else two, else (K > 32) three
+EXPECT_LAUNCHES = {"js_bf16_a": 1 + 1, "js_bf16_staged": 2 + 2, "js_rows288": 4 + 2, "js_k24": 1 + 1, "js_k40": 1 + 3,
+                   "llama8b": 2 + 1}
 
 
 def _run(cfg, impl=binding.IMPL_AUTO, seq_base=0, noise=None):
@@ -33,6 +38,10 @@ def _run(cfg, impl=binding.IMPL_AUTO, seq_base=0, noise=None):
         ctx.set_impl(impl)
         got = to_np(ctx.verify_js(work.H, work.draft, dp, cfg.K, cfg.p, SEED, seq_base=seq_base))
         assert ctx.device_error() == 0
+        LAUNCHES[cfg.name] = ctx.last_launches()
+        again = to_np(ctx.verify_js(work.H, work.draft, dp, cfg.K, cfg.p, SEED, seq_base=seq_base))
+        for key in got:      # the counters the sweeps leave behind are ready for the next call
+            assert np.array_equal(got[key], again[key], equal_nan=got[key].dtype.kind == "f"), key
     finally:
         ctx.close()
     ref = oracle.verify_js(wl.to_numpy_storage(work.W), cfg.dtype, wl.to_numpy_storage(work.H),
@@ -83,6 +92,8 @@ SMALL = [
 def test_js_small_heads(cfg):
     got, ref, draft = _run(cfg, seq_base=3)
     _check(got, ref, draft, cfg)
+    if cfg.name in EXPECT_LAUNCHES:
+        assert LAUNCHES[cfg.name] == EXPECT_LAUNCHES[cfg.name]
     if cfg.K > 1:
         assert ref["js_ok"].any() or ref["js"][..., cfg.K].min() > 0      # the workload is not degenerate
 
@@ -118,6 +129,7 @@ def test_js_needs_its_buffers():
 def test_js_llama8b_full_size():
     cfg = wl.CONFIGS["llama8b"]
     got, ref, draft = _run(cfg)
+    assert LAUNCHES[cfg.name] == EXPECT_LAUNCHES[cfg.name]
     tok_diff = got["tokens"] != ref["tokens"]
     if tok_diff.any():      # full size: allow near-tie flips, judged by the plain oracle's gaps
         work = wl.make_workload(cfg, device="cpu")

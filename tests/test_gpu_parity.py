@@ -180,8 +180,17 @@ def test_tree_against_oracle(ctx, rule):
         check_tree(got, ref, nt, npar, nh, rule)
 
 
-def test_host_entry_point_equals_device_entry_point(ctx):
-    cfg = wl.Config("host", d=256, V=3000, dtype=wl.BF16, B=2, T=5, K=8, p=0.1)
+HOST_CASES = [
+    wl.Config("host", d=256, V=3000, dtype=wl.BF16, B=2, T=5, K=8, p=0.1),      # mask pass reads the pinned H in place
+    wl.Config("host_24", d=256, V=3000, dtype=wl.BF16, B=1, T=3, K=8, p=0.1),   # in-kernel masks: copy kernel first
+    wl.Config("host_f32", d=96, V=1500, dtype=wl.F32, B=2, T=3, K=4, p=0.2),    # CUDA-core head, one finalize block per sequence
+    wl.Config("host_600", d=128, V=2000, dtype=wl.BF16, B=1, T=75, K=8, p=0.1), # several launches, one finalize block
+    wl.Config("host_3x200", d=128, V=2000, dtype=wl.BF16, B=3, T=25, K=8, p=0.1),   # ... and three: the host waits for the stream
+]
+
+
+@pytest.mark.parametrize("cfg", HOST_CASES, ids=lambda c: c.name)
+def test_host_entry_point_equals_device_entry_point(ctx, cfg):
     work = wl.make_workload(cfg, device=DEV)
     ctx.set_head(work.W, max_rows=cfg.rows, max_hidden_rows=cfg.B * cfg.T)
     dev = to_np(ctx.verify_batched(work.H, work.draft, cfg.K, cfg.p, SEED, seq_base=1))
@@ -201,7 +210,7 @@ def test_host_entry_point_equals_device_entry_point(ctx):
     for key in ("tokens", "counts", "hits", "accept_len"):
         assert np.array_equal(host[key].numpy(), dev[key]), key
     with pytest.raises(pk.DropMatchError) as e:
-        big = torch.zeros((cfg.B + 1, cfg.T, cfg.d), dtype=torch.bfloat16)
+        big = torch.zeros((cfg.B + 1, cfg.T, cfg.d), dtype=work.H.dtype)
         ctx.verify_batched_host(big, torch.zeros((cfg.B + 1, cfg.T), dtype=torch.int32), cfg.K, cfg.p, SEED)
     assert e.value.status == binding.EWORKSPACE
 
