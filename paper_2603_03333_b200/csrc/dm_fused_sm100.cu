@@ -60,11 +60,16 @@ constexpr int kPollNs = 32;                 // pause between polls of a barrier 
 constexpr int kIdlePollNs = 500;            // ... and of one that completes once per tile group
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort flag
+// Launch-shape thresholds, in operand rows after padding to 16 (measured on the Llama-3-8B and
+// Qwen3-8B heads; see plan_smem).
 #ifndef DM_PAIR_MIN_NPAD
-#define DM_PAIR_MIN_NPAD 48
+#define DM_PAIR_MIN_NPAD 16     // staged launches at least this wide run as CTA pairs
 #endif
 #ifndef DM_STAGED_MIN_NPAD
-#define DM_STAGED_MIN_NPAD 48   // launches at least this wide are staged even if the slice would fit TMEM as one group
+#define DM_STAGED_MIN_NPAD 16   // slices of several tiles at least this wide are staged even if they would fit TMEM as one group
+#endif
+#ifndef DM_PAIR_PAD_MIN
+#define DM_PAIR_PAD_MIN 64      // narrower pair launches are padded to this many accumulator columns
 #endif
 constexpr int kPairMinNPad = DM_PAIR_MIN_NPAD;   // staged launches at least this wide run as CTA pairs
 
@@ -854,15 +859,18 @@ struct SmemPlan {
 bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     SmemPlan best{};
     int n_pad = (rows + 15) & ~15;
-    // Launches of at least DM_STAGED_MIN_NPAD operand rows are staged even where one group would
-    // fit TMEM (two groups: the first epilogue then overlaps the second group's MMAs), and staged
-    // launches of at least kPairMinNPad rows run as CTA pairs: half the MMA issue work and half
-    // the operand bytes per SM.  Measured faster than lone CTAs, and than the one-group mode with
-    // its in-kernel Philox builders, from 33 paths up (equal on boxes that hold their clock, 4-25 us
-    // faster on boxes that the power cap slows down).
+    // A slice of several tiles is staged even where it would fit TMEM as one group (single-tile
+    // groups: all but the last tile's epilogue overlaps the MMAs that follow), and staged launches
+    // run as CTA pairs: half the MMA issue work and half the operand bytes per SM.  Measured faster
+    // than lone CTAs, and than the one-group mode with its in-kernel Philox builders, at every
+    // path count (Llama-3-8B head, 8-32 paths: 157 against 163 us per call; Qwen3-8B: 188 against
+    // 193 us), so the builders are left with the heads whose slices are a single tile.  Pair
+    // launches narrower than 64 accumulator columns are padded to 64 (N = 32 MMAs were 6 us slower
+    // on the Llama-3-8B head); the columns past the call's paths are computed and ignored.
     const bool force_staged = n_pad >= DM_STAGED_MIN_NPAD && tiles_per_cta > 1;
     best.pair = ((tiles_per_cta > kTmemCols / n_pad || force_staged) && n_pad >= kPairMinNPad) ? 1 : 0;
     if (best.pair) n_pad = (rows + 31) & ~31;
+    if (best.pair && n_pad < DM_PAIR_PAD_MIN) n_pad = DM_PAIR_PAD_MIN;
     best.n_pad = n_pad;
     best.n_slots = kTmemCols / n_pad;
     const uint32_t b_stage = (uint32_t)(best.pair ? n_pad / 2 : n_pad) * (kBlockK * 2);
@@ -981,7 +989,9 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
     const bool two_staged = max_rows > kMaxNPad && plan_smem(kMaxNPad, fs->geo[1].tiles_per_cta, &plan_two) &&
                             plan_two.staged;
     if (plan.staged || two_staged) {
-        fs->staging_rows = (max_rows + 15) & ~15;
+        // room for the widest box a launch may ask for: a padded pair launch reads 2 x 32 rows
+        fs->staging_rows = (max_rows + 31) & ~31;
+        if (fs->staging_rows < DM_PAIR_PAD_MIN) fs->staging_rows = DM_PAIR_PAD_MIN;
         const size_t n = (size_t)fs->staging_rows * head.d * sizeof(__nv_bfloat16);
         if (cudaMalloc(&fs->staging, n) != cudaSuccess) { cudaGetLastError(); delete fs; return DM_ECUDA; }
         if (cudaMemset(fs->staging, 0, n) != cudaSuccess) { cudaGetLastError(); cudaFree(fs->staging); delete fs; return DM_ECUDA; }

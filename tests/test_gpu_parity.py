@@ -292,6 +292,11 @@ EDGE = [
     wl.Config("edge_rows257", d=64, V=1000, dtype=wl.BF16, B=1, T=1, K=257, p=0.1),
     # a vocabulary so large that a slice has 16 tiles even at 24 paths (staged operand, many groups)
     wl.Config("edge_big_v", d=64, V=300000, dtype=wl.BF16, B=1, T=3, K=8, p=0.1),
+    # 1, 8 and 24 paths on a head whose slices have several tiles: CTA pairs padded to 64 accumulator
+    # columns, with a staging buffer sized for nothing wider
+    wl.Config("edge_pad_r1", d=128, V=60000, dtype=wl.BF16, B=1, T=1, K=1, p=0.2),
+    wl.Config("edge_pad_r8", d=128, V=60000, dtype=wl.BF16, B=1, T=1, K=8, p=0.2),
+    wl.Config("edge_pad_r24", d=192, V=50000, dtype=wl.BF16, B=1, T=3, K=8, p=0.1),
     # a long hidden size (256 blocks of 64) on a small vocabulary
     wl.Config("edge_long_d", d=16384, V=700, dtype=wl.BF16, B=1, T=2, K=8, p=0.1),
     # fp32 head whose hidden size is the minimum the CUDA-core kernel takes
