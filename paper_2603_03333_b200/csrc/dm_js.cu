@@ -1,11 +1,16 @@
 // JS-divergence acceptance (Sec. 3.2: Eq. 4 centroid, Eq. 5 test, Algorithm 1) on the logits that
-// a head kernel has written to global memory.  Three small kernels over [n_pos][K][V] fp32
-// logits (20 MB for the Llama-3-8B head at 40 paths, L2-resident right after the head kernel):
-//   js_lse_kernel      per (position, vocabulary chunk): partial log-sum-exp of each of the K
-//                      paths and of the centroid logits (their mean over the paths)
-//   js_sum_kernel      per (position, chunk): merges the partial log-sum-exps, then the chunk's
-//                      share of JS(p_i || pbar) for every path and of JS(phat || pbar)
-//   js_accept_kernel   per sequence: sums the shares, Eq. 5, else Eq. 6, left-to-right scan
+// a head kernel has written to global memory: [n_pos][K][V] fp32 (20 MB for the Llama-3-8B head at
+// 40 paths; the head kernel streams W with an evict-first policy, so they are still in L2).
+// Up to 32 paths per position, js_sweep_kernel does the work, a block per (position, vocabulary
+// chunk) that holds its chunk in shared memory:
+//   first sweep    the chunk's part of the log-sum-exp of each of the K paths and of the centroid
+//                  logits (their mean over the paths); the last block of a position to finish
+//                  merges the parts
+//   second sweep   the chunk's share of JS(p_i || pbar) for every path and of JS(phat || pbar);
+//                  the last block of the grid sums the shares and runs Algorithm 1 and the scan
+// either as one cooperative launch (calls whose logits fit the shared memory of the GPU: the
+// chunk stays where it is between the sweeps) or as two launches.  More paths than that: three
+// plain kernels that take one series at a time (js_lse_kernel, js_sum_kernel, js_accept_kernel).
 // Probabilities are never stored: p = exp(l - lse) is recomputed where it is needed.
 #include "dm_finalize.cuh"
 #include "dm_internal.h"
@@ -169,149 +174,18 @@ __device__ __forceinline__ void js_accept_sequence(const JsAcceptArgs& a, int b,
     __syncthreads();
 }
 
-// ---- the same two sweeps for K <= KMAX paths with every series kept in registers --------------
-// A thread takes vocabulary entries v0 + tid, v0 + tid + 256, ...: it loads the K logits of an
-// entry once (coalesced across the block), forms the centroid and updates all K+1 running
-// results; the block is reduced once at the end.  Slot KMAX holds the centroid (first sweep) or
-// the draft distribution (second sweep).
-
-__device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
-    const float M = fmaxf(m, m2);
-    if (M == -INFINITY) { m = M; s = 0.0f; return; }
-    // fast exponentials: relative error ~1e-7 per term of a sum of positive terms, far inside the
-    // tolerance of the divergences (the arguments are <= 0)
-    s = s * __expf(m - M) + s2 * __expf(m2 - M);
-    m = M;
-}
-
-template <int KMAX>
-__global__ void __launch_bounds__(kJsThreads)
-js_lse_reg_kernel(const float* __restrict__ logits, int V, int K, int chunk_len, int n_chunks,
-                  float2* __restrict__ part) {
-    __shared__ float2 red[kJsThreads / 32][KMAX + 1];
-    const int pos = blockIdx.y, chunk = blockIdx.x;
-    const int v0 = chunk * chunk_len, v1 = min(V, v0 + chunk_len);
-    const float* pl = logits + (size_t)pos * K * V;
-    float m[KMAX + 1], s[KMAX + 1];
-#pragma unroll
-    for (int i = 0; i <= KMAX; ++i) { m[i] = -INFINITY; s[i] = 0.0f; }
-    const float inv_k = 1.0f / (float)K;
-    for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) {
-        float c = 0.0f;
-#pragma unroll
-        for (int i = 0; i < KMAX; ++i)
-            if (i < K) {
-                const float x = pl[(size_t)i * V + v];
-                c += x;
-                lse_merge(m[i], s[i], x, 1.0f);
-            }
-        lse_merge(m[KMAX], s[KMAX], c * inv_k, 1.0f);
-    }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#pragma unroll
-    for (int i = 0; i <= KMAX; ++i) {
-        if (i < K || i == KMAX) {
-            float M = m[i];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
-            float t = M == -INFINITY ? 0.0f : s[i] * __expf(m[i] - M);   // one rescale, then a plain sum
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
-            if (lane == 0) red[warp][i] = make_float2(M, t);
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i <= KMAX; i += kJsThreads) {
-        if (i < K || i == KMAX) {
-            float mm = red[0][i].x, ss = red[0][i].y;
-            for (int w = 1; w < kJsThreads / 32; ++w) lse_merge(mm, ss, red[w][i].x, red[w][i].y);
-            const int series = i == KMAX ? K : i;
-            part[((size_t)pos * (K + 1) + series) * n_chunks + chunk] = make_float2(mm, ss);
-        }
-    }
-}
-
-// The block that finishes last (a ticket counter in global memory, left at zero) also runs
-// Algorithm 1 and the scan for every sequence: no third kernel.
-template <int KMAX>
-__global__ void __launch_bounds__(kJsThreads)
-js_sum_reg_kernel(const float* __restrict__ logits, const float* __restrict__ draft_prob, int V, int K,
-                  int chunk_len, int n_chunks, const float2* __restrict__ part, float* __restrict__ share,
-                  unsigned int* __restrict__ ticket, JsAcceptArgs accept) {
-    extern __shared__ int32_t ok_scratch[];   // [T], for the last block
-    __shared__ unsigned int s_ticket;
-    __shared__ float lse[KMAX + 1];
-    __shared__ float red[kJsThreads / 32][KMAX + 1];
-    const int pos = blockIdx.y, chunk = blockIdx.x;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int series = warp; series <= K; series += kJsThreads / 32) {   // merge the chunks' partial log-sum-exps
-        const float2* ps = part + ((size_t)pos * (K + 1) + series) * n_chunks;
-        float mm = -INFINITY, ss = 0.0f;
-        for (int c = lane; c < n_chunks; c += 32) lse_merge(mm, ss, ps[c].x, ps[c].y);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1)
-            lse_merge(mm, ss, __shfl_xor_sync(0xFFFFFFFFu, mm, off), __shfl_xor_sync(0xFFFFFFFFu, ss, off));
-        if (lane == 0) lse[series == K ? KMAX : series] = mm + logf(ss);
-    }
-    __syncthreads();
-    const int v0 = chunk * chunk_len, v1 = min(V, v0 + chunk_len);
-    const float* pl = logits + (size_t)pos * K * V;
-    const float* dp = draft_prob + (size_t)pos * V;
-    float acc[KMAX + 1];
-#pragma unroll
-    for (int i = 0; i <= KMAX; ++i) acc[i] = 0.0f;
-    const float inv_k = 1.0f / (float)K, lse_c = lse[KMAX];
-    for (int v = v0 + threadIdx.x; v < v1; v += kJsThreads) {
-        float x[KMAX];
-        float c = 0.0f;
-#pragma unroll
-        for (int i = 0; i < KMAX; ++i)
-            if (i < K) { x[i] = pl[(size_t)i * V + v]; c += x[i]; }
-        const float lq = c * inv_k - lse_c;                       // log pbar[v]
-#pragma unroll
-        for (int i = 0; i < KMAX; ++i)
-            if (i < K) acc[i] += js_term(x[i] - lse[i], lq);
-        const float P = dp[v];
-        acc[KMAX] += js_term(P > 0.0f ? logf(P) : -INFINITY, lq);
-    }
-#pragma unroll
-    for (int i = 0; i <= KMAX; ++i) {
-        if (i < K || i == KMAX) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc[i] += __shfl_xor_sync(0xFFFFFFFFu, acc[i], off);
-            if (lane == 0) red[warp][i] = acc[i];
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i <= KMAX; i += kJsThreads) {
-        if (i < K || i == KMAX) {
-            float t = 0.0f;
-            for (int w = 0; w < kJsThreads / 32; ++w) t += red[w][i];
-            const int series = i == KMAX ? K : i;
-            share[((size_t)pos * (K + 1) + series) * n_chunks + chunk] = 0.5f * t;
-        }
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_ticket = atomicAdd(ticket, 1u);
-    __syncthreads();
-    if (s_ticket == gridDim.x * gridDim.y - 1) {
-        __threadfence();
-        for (int b = 0; b < accept.B; ++b) js_accept_sequence(accept, b, ok_scratch);
-        if (threadIdx.x == 0) *ticket = 0u;
-    }
-}
-
-// ---- both sweeps in one kernel, for calls whose logits fit the shared memory of the GPU ---------
-// Launched cooperatively (every block resident).  A block copies its chunk of the K logit rows
-// of its position and of the draft distribution into shared memory (asynchronous copies, all in
-// flight at once), adds the centroid logits (Eq. 4 before the softmax) as one more row, and forms
-// its part of every log-sum-exp from the chunk's own maxima.  The blocks of a position then meet
-// at a counter in global memory (bounded waits): the last to arrive merges the parts and
-// publishes the K+1 log-sum-exps, the others wait for its flag.  Every block then forms its share
-// of the divergences from the copy in shared memory: the logits cross the memory system once,
-// and there is one launch.  The last block of the grid runs Algorithm 1 and leaves the counters
-// at zero.
+// ---- the two sweeps for up to 32 paths per position ---------------------------------------------
+// A block copies its chunk of the K logit rows of its position and of the draft distribution
+// into shared memory (asynchronous copies, all in flight at once) and adds the centroid logits
+// (Eq. 4 before the softmax) as one more row.
+// MODE 0: both sweeps.  Launched cooperatively (every block resident): after the first sweep the
+//         blocks of a position meet at a counter in global memory (bounded waits); the last to
+//         arrive merges the parts and publishes the K+1 log-sum-exps, the others wait for its
+//         flag; the second sweep then runs on the copy in shared memory: the logits cross the
+//         memory system once, and there is one launch.
+// MODE 1: the first sweep alone (nobody waits: the last block of a position merges).
+// MODE 2: the second sweep alone, on a fresh copy, with the log-sum-exps that MODE 1 published.
+// In modes 0 and 2 the last block of the grid runs Algorithm 1 and leaves the counters at zero.
 __device__ __forceinline__ float ex2_fast(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -403,12 +277,12 @@ __device__ __forceinline__ void js_accept_staged(const JsAcceptArgs& a, float* s
 
 // words: [0] ticket of the grid, [1 + pos] arrivals of a position, [1 + n_pos + pos] "log-sum-exps
 // published" flag of a position; lse_out[pos][K+1] in global memory.
-template <int KMAX>
+template <int KMAX, int MODE>
 __global__ void __launch_bounds__(kJsThreads)
-js_one_kernel(const float* __restrict__ logits, const float* __restrict__ draft_prob, int V, int K, int chunk_len,
-              int n_chunks, int vec, float2* __restrict__ part, float* __restrict__ share, float* __restrict__ lse_out,
-              unsigned int* __restrict__ words, long long wait_limit, uint32_t* __restrict__ err, int scratch_floats,
-              JsAcceptArgs accept) {
+js_sweep_kernel(const float* __restrict__ logits, const float* __restrict__ draft_prob, int V, int K, int chunk_len,
+                int n_chunks, int vec, float2* __restrict__ part, float* __restrict__ share, float* __restrict__ lse_out,
+                unsigned int* __restrict__ words, long long wait_limit, uint32_t* __restrict__ err, int scratch_floats,
+                JsAcceptArgs accept) {
     extern __shared__ __align__(16) float xs[];   // [K+2][chunk_len]: logits, centroid logits, draft probabilities
     __shared__ unsigned int s_ticket, s_last;
     __shared__ float bm[KMAX + 1], lse[KMAX + 1];
@@ -421,14 +295,15 @@ js_one_kernel(const float* __restrict__ logits, const float* __restrict__ draft_
     float* xc = xs + (size_t)K * chunk_len;         // centroid row
     float* xd = xs + (size_t)(K + 1) * chunk_len;   // draft row
     // ---- copy the chunk: every load of the block in flight at once
+    const int n_rows = MODE == 1 ? K : K + 1;       // the first sweep alone has no use for the draft row
     if (vec) {
-        for (int i = 0; i <= K; ++i) {
+        for (int i = 0; i < n_rows; ++i) {
             const float* src = i < K ? pl + (size_t)i * V : dp;
             float* dst = i < K ? xs + (size_t)i * chunk_len : xd;
             for (int x = 4 * threadIdx.x; x < n; x += 4 * kJsThreads) cp_async_f4(dst + x, src + x);
         }
     } else {
-        for (int i = 0; i <= K; ++i) {
+        for (int i = 0; i < n_rows; ++i) {
             const float* src = i < K ? pl + (size_t)i * V : dp;
             float* dst = i < K ? xs + (size_t)i * chunk_len : xd;
             for (int x = threadIdx.x; x < n; x += kJsThreads) cp_async_f1(dst + x, src + x);
@@ -437,7 +312,7 @@ js_one_kernel(const float* __restrict__ logits, const float* __restrict__ draft_
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
-    // ---- first sweep: centroid logits and the chunk's maxima, then the sums of exponentials
+    // ---- centroid logits (and, for the first sweep, the chunk's maxima)
     const float inv_k = 1.0f / (float)K;
     float mx[KMAX + 1];
 #pragma unroll
@@ -455,106 +330,112 @@ js_one_kernel(const float* __restrict__ logits, const float* __restrict__ draft_
         xc[x] = c;
         mx[KMAX] = fmaxf(mx[KMAX], c);
     }
-#pragma unroll
-    for (int i = 0; i <= KMAX; ++i)
-        if (i < K || i == KMAX) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xFFFFFFFFu, mx[i], off));
-            if (lane == 0) red[warp][i] = mx[i];
-        }
-    __syncthreads();
-    for (int i = threadIdx.x; i <= KMAX; i += kJsThreads)
-        if (i < K || i == KMAX) {
-            float t = red[0][i];
-            for (int w = 1; w < kJsThreads / 32; ++w) t = fmaxf(t, red[w][i]);
-            bm[i] = t;   // (-inf for an empty chunk)
-        }
-    __syncthreads();
     float acc[KMAX + 1];
+    if (MODE != 2) {
+        // ---- first sweep: the sums of exponentials around the chunk's maxima
 #pragma unroll
-    for (int i = 0; i <= KMAX; ++i) acc[i] = 0.0f;
-    for (int x = threadIdx.x; x < n; x += kJsThreads) {    // the thread reads back its own centroid entries
+        for (int i = 0; i <= KMAX; ++i)
+            if (i < K || i == KMAX) {
 #pragma unroll
-        for (int i = 0; i < KMAX; ++i)
-            if (i < K) acc[i] += ex2_fast((xs[i * chunk_len + x] - bm[i]) * kLog2e);
-        acc[KMAX] += ex2_fast((xc[x] - bm[KMAX]) * kLog2e);
-    }
-#pragma unroll
-    for (int i = 0; i <= KMAX; ++i)
-        if (i < K || i == KMAX) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc[i] += __shfl_xor_sync(0xFFFFFFFFu, acc[i], off);
-            if (lane == 0) red[warp][i] = acc[i];
-        }
-    __syncthreads();
-    for (int i = threadIdx.x; i <= KMAX; i += kJsThreads)
-        if (i < K || i == KMAX) {
-            float t = 0.0f;
-            for (int w = 0; w < kJsThreads / 32; ++w) t += red[w][i];
-            part[((size_t)pos * (K + 1) + (i == KMAX ? K : i)) * n_chunks + chunk] = make_float2(bm[i], t);
-            __threadfence();
-        }
-    __syncthreads();
-    // ---- the blocks of this position meet
-    if (threadIdx.x == 0) s_last = atomicAdd(words + 1 + pos, 1u) == (unsigned int)(n_chunks - 1) ? 1u : 0u;
-    __syncthreads();
-    if (s_last) {
-        // the last to arrive: every part of this position is in global memory
-        __threadfence();
-        // a half-warp per series: its loads all in flight, then the maximum, then one rescaled sum
-        const int hw = threadIdx.x >> 4, hl = threadIdx.x & 15;
-        for (int s0 = 0; s0 <= K; s0 += kJsThreads / 16) {
-            const int series = s0 + hw;
-            const bool valid = series <= K;
-            const float2* ps = part + ((size_t)pos * (K + 1) + (valid ? series : 0)) * n_chunks;
-            float mm = -INFINITY, ss = 0.0f;
-            for (int c0 = 0; c0 < n_chunks; c0 += 128) {
-                float2 pr[8];
-                float m8 = -INFINITY;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int c = c0 + 16 * u + hl;
-                    pr[u] = (valid && c < n_chunks) ? __ldcg(ps + c) : make_float2(-INFINITY, 0.0f);
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) m8 = fmaxf(m8, pr[u].x);
-                const float M = fmaxf(mm, m8);
-                float t = ss == 0.0f ? 0.0f : ss * ex2_fast((mm - M) * kLog2e);
-#pragma unroll
-                for (int u = 0; u < 8; ++u) t += pr[u].y == 0.0f ? 0.0f : pr[u].y * ex2_fast((pr[u].x - M) * kLog2e);
-                mm = M;
-                ss = t;
+                for (int off = 16; off > 0; off >>= 1) mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xFFFFFFFFu, mx[i], off));
+                if (lane == 0) red[warp][i] = mx[i];
             }
-            float M = mm;
+        __syncthreads();
+        for (int i = threadIdx.x; i <= KMAX; i += kJsThreads)
+            if (i < K || i == KMAX) {
+                float t = red[0][i];
+                for (int w = 1; w < kJsThreads / 32; ++w) t = fmaxf(t, red[w][i]);
+                bm[i] = t;   // (-inf for an empty chunk)
+            }
+        __syncthreads();
 #pragma unroll
-            for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
-            float t = ss == 0.0f ? 0.0f : ss * ex2_fast((mm - M) * kLog2e);
+        for (int i = 0; i <= KMAX; ++i) acc[i] = 0.0f;
+        for (int x = threadIdx.x; x < n; x += kJsThreads) {    // the thread reads back its own centroid entries
 #pragma unroll
-            for (int off = 8; off > 0; off >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
-            if (valid && hl == 0) {
-                const float l = M + logf(t);
-                lse[series == K ? KMAX : series] = l;
-                lse_out[(size_t)pos * (K + 1) + series] = l;
+            for (int i = 0; i < KMAX; ++i)
+                if (i < K) acc[i] += ex2_fast((xs[i * chunk_len + x] - bm[i]) * kLog2e);
+            acc[KMAX] += ex2_fast((xc[x] - bm[KMAX]) * kLog2e);
+        }
+#pragma unroll
+        for (int i = 0; i <= KMAX; ++i)
+            if (i < K || i == KMAX) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc[i] += __shfl_xor_sync(0xFFFFFFFFu, acc[i], off);
+                if (lane == 0) red[warp][i] = acc[i];
+            }
+        __syncthreads();
+        for (int i = threadIdx.x; i <= KMAX; i += kJsThreads)
+            if (i < K || i == KMAX) {
+                float t = 0.0f;
+                for (int w = 0; w < kJsThreads / 32; ++w) t += red[w][i];
+                part[((size_t)pos * (K + 1) + (i == KMAX ? K : i)) * n_chunks + chunk] = make_float2(bm[i], t);
                 __threadfence();
             }
-        }
         __syncthreads();
-        if (threadIdx.x == 0) atomicExch(words + 1 + n_pos + pos, 1u);
-    } else {
-        if (threadIdx.x == 0) {
-            volatile unsigned int* flag = words + 1 + n_pos + pos;
-            const long long t0 = clock64();
-            unsigned int seen = 0u;
-            while ((seen = *flag) == 0u) {
-                if (clock64() - t0 > wait_limit) {     // give up: the call then accepts nothing (the error word is set)
-                    atomicCAS(err, 0u, (uint32_t)ERR_WAIT_JS);
-                    break;
-                }
-                __nanosleep(32);
-            }
+        // ---- the blocks of this position meet
+        if (threadIdx.x == 0) s_last = atomicAdd(words + 1 + pos, 1u) == (unsigned int)(n_chunks - 1) ? 1u : 0u;
+        __syncthreads();
+        if (s_last) {
+            // the last to arrive: every part of this position is in global memory
             __threadfence();
+            // a half-warp per series: its loads all in flight, then the maximum, then one rescaled sum
+            const int hw = threadIdx.x >> 4, hl = threadIdx.x & 15;
+            for (int s0 = 0; s0 <= K; s0 += kJsThreads / 16) {
+                const int series = s0 + hw;
+                const bool valid = series <= K;
+                const float2* ps = part + ((size_t)pos * (K + 1) + (valid ? series : 0)) * n_chunks;
+                float mm = -INFINITY, ss = 0.0f;
+                for (int c0 = 0; c0 < n_chunks; c0 += 128) {
+                    float2 pr[8];
+                    float m8 = -INFINITY;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int c = c0 + 16 * u + hl;
+                        pr[u] = (valid && c < n_chunks) ? __ldcg(ps + c) : make_float2(-INFINITY, 0.0f);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) m8 = fmaxf(m8, pr[u].x);
+                    const float M = fmaxf(mm, m8);
+                    float t = ss == 0.0f ? 0.0f : ss * ex2_fast((mm - M) * kLog2e);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) t += pr[u].y == 0.0f ? 0.0f : pr[u].y * ex2_fast((pr[u].x - M) * kLog2e);
+                    mm = M;
+                    ss = t;
+                }
+                float M = mm;
+#pragma unroll
+                for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, off));
+                float t = ss == 0.0f ? 0.0f : ss * ex2_fast((mm - M) * kLog2e);
+#pragma unroll
+                for (int off = 8; off > 0; off >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, off);
+                if (valid && hl == 0) {
+                    const float l = M + logf(t);
+                    lse[series == K ? KMAX : series] = l;
+                    lse_out[(size_t)pos * (K + 1) + series] = l;
+                    __threadfence();
+                }
+            }
+            __syncthreads();
+            if (MODE == 0 && threadIdx.x == 0) atomicExch(words + 1 + n_pos + pos, 1u);
+        } else if (MODE == 0) {
+            if (threadIdx.x == 0) {
+                volatile unsigned int* flag = words + 1 + n_pos + pos;
+                const long long t0 = clock64();
+                while (*flag == 0u) {
+                    if (clock64() - t0 > wait_limit) {     // give up: the call then accepts nothing (the error word is set)
+                        atomicCAS(err, 0u, (uint32_t)ERR_WAIT_JS);
+                        break;
+                    }
+                    __nanosleep(32);
+                }
+                __threadfence();
+            }
+            __syncthreads();
+            for (int i = threadIdx.x; i <= K; i += kJsThreads) lse[i == K ? KMAX : i] = __ldcg(lse_out + (size_t)pos * (K + 1) + i);
+            __syncthreads();
         }
-        __syncthreads();
+        if (MODE == 1) return;
+    } else {
         for (int i = threadIdx.x; i <= K; i += kJsThreads) lse[i == K ? KMAX : i] = __ldcg(lse_out + (size_t)pos * (K + 1) + i);
         __syncthreads();
     }
@@ -619,8 +500,9 @@ int js_chunks(int V, int n_pos) {
 }
 
 size_t js_words_offset(int V, int max_rows, int max_hidden) {
-    // partial (max, sum) pairs and JS shares for every (position, series, chunk), at the largest chunk count
-    return (size_t)(max_rows + max_hidden) * ((V + 1023) / 1024) * 3;
+    // partial (max, sum) pairs and JS shares for every (position, series, chunk), at the largest
+    // chunk count (chunks of 512 entries, which the two-launch form takes from 17 paths up)
+    return (size_t)(max_rows + max_hidden) * ((V + 511) / 512) * 3;
 }
 
 size_t js_workspace_floats(int V, int max_rows, int max_hidden) {
@@ -631,27 +513,33 @@ size_t js_workspace_floats(int V, int max_rows, int max_hidden) {
 
 namespace {
 
-// Both sweeps as one cooperative launch, if the call's logits fit the shared memory of the SMs with
-// every block resident.  Returns DM_EUNSUPPORTED if they do not (the caller then runs two kernels).
+// The two sweeps for K <= KMAX: one cooperative launch if the call's logits fit the shared memory of
+// the SMs with every block resident, else two plain launches with chunks of about 1024 entries.
 template <int KMAX>
-int launch_js_one(const float* logits, const float* draft_prob, float* workspace, float* lse_out, unsigned int* words, int V,
-                  int n_pos, int K, int T, const JsAcceptArgs& acc_in, long long wait_limit, uint32_t* err,
-                  cudaStream_t stream) {
+int launch_js_sweeps(const float* logits, const float* draft_prob, float* workspace, float* lse_out, unsigned int* words,
+                     int V, int n_pos, int K, int T, const JsAcceptArgs& acc_in, long long wait_limit, uint32_t* err,
+                     cudaStream_t stream, int* launches_out) {
     int sms = 148, dev = 0, coop = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return DM_ECUDA;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (!coop) return DM_EUNSUPPORTED;
     static bool attr_set = false;
     const int smem_cap = 200 * 1024;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(js_one_kernel<KMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess) {
+        if (cudaFuncSetAttribute(js_sweep_kernel<KMAX, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(js_sweep_kernel<KMAX, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(js_sweep_kernel<KMAX, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess) {
             cudaGetLastError();
-            return DM_EUNSUPPORTED;
+            return DM_ECUDA;
         }
         attr_set = true;
     }
-    for (int per_sm = 4; per_sm >= 1; --per_sm) {   // more resident blocks hide more latency
+    float2* part = reinterpret_cast<float2*>(workspace);
+    JsAcceptArgs acc = acc_in;
+    // 16-byte copies where every row of every chunk starts on a 16-byte boundary
+    int vec = (V % 4 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15u) == 0 &&
+               (reinterpret_cast<uintptr_t>(draft_prob) & 15u) == 0) ? 1 : 0;
+    for (int per_sm = coop ? 4 : 0; per_sm >= 1; --per_sm) {   // more resident blocks hide more latency
         int n_chunks = (V + 1023) / 1024;
         const int fit = (per_sm * sms) / n_pos;
         if (n_chunks > fit) n_chunks = fit;
@@ -661,32 +549,44 @@ int launch_js_one(const float* logits, const float* draft_prob, float* workspace
         if (smem < (size_t)T * sizeof(int32_t)) smem = (size_t)T * sizeof(int32_t);
         if (smem > (size_t)smem_cap) continue;
         int resident = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, js_one_kernel<KMAX>, kJsThreads, smem) != cudaSuccess) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, js_sweep_kernel<KMAX, 0>, kJsThreads, smem) != cudaSuccess) {
             cudaGetLastError();
-            return DM_EUNSUPPORTED;
+            break;
         }
         if ((long long)resident * sms < (long long)n_chunks * n_pos) continue;
-        float2* part = reinterpret_cast<float2*>(workspace);
         float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
-        JsAcceptArgs acc = acc_in;
         acc.share = share;
         acc.n_chunks = n_chunks;
-        // 16-byte copies where every row of every chunk starts on a 16-byte boundary
-        int vec = (V % 4 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15u) == 0 &&
-                   (reinterpret_cast<uintptr_t>(draft_prob) & 15u) == 0) ? 1 : 0;
         int scratch_floats = (int)(smem / sizeof(float));
         void* args[] = {(void*)&logits, (void*)&draft_prob, (void*)&V, (void*)&K, (void*)&chunk_len, (void*)&n_chunks,
                         (void*)&vec, (void*)&part, (void*)&share, (void*)&lse_out, (void*)&words, (void*)&wait_limit,
                         (void*)&err, (void*)&scratch_floats, (void*)&acc};
-        if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(js_one_kernel<KMAX>),
+        if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(js_sweep_kernel<KMAX, 0>),
                                         dim3((unsigned)n_chunks, (unsigned)n_pos), dim3(kJsThreads), args, smem,
                                         stream) != cudaSuccess) {
             cudaGetLastError();
             return DM_ECUDA;
         }
+        *launches_out = 1;
         return DM_OK;
     }
-    return DM_EUNSUPPORTED;
+    // Two launches.  Chunks of 1024 entries, 512 from 17 paths up (two blocks per SM either way).
+    const int chunk_len = KMAX <= 16 ? 1024 : 512;
+    int n_chunks = (V + chunk_len - 1) / chunk_len;
+    size_t smem = (size_t)(K + 2) * chunk_len * sizeof(float);
+    if (smem < (size_t)T * sizeof(int32_t)) smem = (size_t)T * sizeof(int32_t);
+    if (smem > (size_t)smem_cap) return DM_EUNSUPPORTED;
+    float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
+    acc.share = share;
+    acc.n_chunks = n_chunks;
+    const int scratch_floats = (int)(smem / sizeof(float));
+    const dim3 grid((unsigned)n_chunks, (unsigned)n_pos);
+    js_sweep_kernel<KMAX, 1><<<grid, kJsThreads, smem, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, vec, part,
+                                                              share, lse_out, words, wait_limit, err, scratch_floats, acc);
+    js_sweep_kernel<KMAX, 2><<<grid, kJsThreads, smem, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, vec, part,
+                                                              share, lse_out, words, wait_limit, err, scratch_floats, acc);
+    *launches_out = 2;
+    return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 
 }  // namespace
@@ -694,45 +594,35 @@ int launch_js_one(const float* logits, const float* draft_prob, float* workspace
 int launch_js(const float* logits, const float* draft_prob, float* workspace, size_t words_offset, int max_hidden, int V, int B, int T,
               int K, const int32_t* tokens, const int32_t* draft, float* out_js, int32_t* out_js_ok,
               int32_t* out_accept_len, uint32_t* err, long long wait_limit, cudaStream_t stream, int* launches_out) {
-    const int n_pos = B * T, n_chunks = js_chunks(V, n_pos);
+    const int n_pos = B * T;
     if (n_pos > kJsMaxPositions) return DM_EUNSUPPORTED;   // positions are the grid's second dimension
-    const size_t ticket_offset = words_offset;
-    if (launches_out) *launches_out = 1;
-    if (K <= 32) {   // small calls: both sweeps in one launch, the logits held in shared memory in between
+    int launches = 0;
+    if (K <= 32) {
         unsigned int* words = reinterpret_cast<unsigned int*>(workspace + words_offset);
         float* lse_out = workspace + words_offset + 4 + 2 * (size_t)max_hidden;
         const JsAcceptArgs a1{nullptr, 0, B, T, K, tokens, draft, out_js, out_js_ok, out_accept_len, err};
         const long long limit = wait_limit > 0 ? wait_limit : 2000000000ll;
-        const int st = K <= 8    ? launch_js_one<8>(logits, draft_prob, workspace, lse_out, words, V, n_pos, K, T, a1, limit, err, stream)
-                       : K <= 16 ? launch_js_one<16>(logits, draft_prob, workspace, lse_out, words, V, n_pos, K, T, a1, limit, err, stream)
-                                 : launch_js_one<32>(logits, draft_prob, workspace, lse_out, words, V, n_pos, K, T, a1, limit, err, stream);
-        if (st != DM_EUNSUPPORTED) return st;
+        const int st = K <= 8    ? launch_js_sweeps<8>(logits, draft_prob, workspace, lse_out, words, V, n_pos, K, T, a1, limit, err, stream, &launches)
+                       : K <= 16 ? launch_js_sweeps<16>(logits, draft_prob, workspace, lse_out, words, V, n_pos, K, T, a1, limit, err, stream, &launches)
+                                 : launch_js_sweeps<32>(logits, draft_prob, workspace, lse_out, words, V, n_pos, K, T, a1, limit, err, stream, &launches);
+        if (launches_out) *launches_out = launches;
+        return st;
     }
-    if (launches_out) *launches_out = K <= 32 ? 2 : 3;
+    // More paths than the sweep kernel keeps in registers: one series at a time, acceptance in a kernel of its own.
+    if (launches_out) *launches_out = 3;
+    const int n_chunks = js_chunks(V, n_pos);
     const int chunk_len = (V + n_chunks - 1) / n_chunks;
     float2* part = reinterpret_cast<float2*>(workspace);
     float* share = workspace + (size_t)n_pos * (K + 1) * n_chunks * 2;
-    unsigned int* ticket = reinterpret_cast<unsigned int*>(workspace + ticket_offset);
     if ((size_t)(K + 1 + chunk_len) * sizeof(float) > 40 * 1024 || (size_t)T * sizeof(int32_t) > 40 * 1024) return DM_EUNSUPPORTED;
     dim3 grid((unsigned)n_chunks, (unsigned)n_pos);
     const JsAcceptArgs acc{share, n_chunks, B, T, K, tokens, draft, out_js, out_js_ok, out_accept_len, err};
     const size_t ok_bytes = (size_t)T * sizeof(int32_t);
-    if (K <= 8) {
-        js_lse_reg_kernel<8><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_reg_kernel<8><<<grid, kJsThreads, ok_bytes, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share, ticket, acc);
-    } else if (K <= 16) {
-        js_lse_reg_kernel<16><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_reg_kernel<16><<<grid, kJsThreads, ok_bytes, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share, ticket, acc);
-    } else if (K <= 32) {
-        js_lse_reg_kernel<32><<<grid, kJsThreads, 0, stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_reg_kernel<32><<<grid, kJsThreads, ok_bytes, stream>>>(logits, draft_prob, V, K, chunk_len, n_chunks, part, share, ticket, acc);
-    } else {   // more paths than fit in registers: one series at a time, acceptance in a kernel of its own
-        js_lse_kernel<<<grid, kJsThreads, chunk_len * sizeof(float), stream>>>(logits, V, K, chunk_len, n_chunks, part);
-        js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K,
-                                                                                      chunk_len, n_chunks, part, share);
-        if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
-        js_accept_kernel<<<B, kJsThreads, ok_bytes, stream>>>(acc);
-    }
+    js_lse_kernel<<<grid, kJsThreads, chunk_len * sizeof(float), stream>>>(logits, V, K, chunk_len, n_chunks, part);
+    js_sum_kernel<<<grid, kJsThreads, (K + 1 + chunk_len) * sizeof(float), stream>>>(logits, draft_prob, V, K,
+                                                                                  chunk_len, n_chunks, part, share);
+    if (cudaGetLastError() != cudaSuccess) return DM_ECUDA;
+    js_accept_kernel<<<B, kJsThreads, ok_bytes, stream>>>(acc);
     return cudaGetLastError() == cudaSuccess ? DM_OK : DM_ECUDA;
 }
 
