@@ -150,11 +150,12 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
         ev_end = c->prof_events[c->prof_used + 1];
         cudaEventRecord(ev_begin, stream);
     }
-    bool folded = false;
+    bool folded = false, best_reduced = false;
+    unsigned long long* best = c->partials + (size_t)kMaxSlices * c->max_rows;   // one word per path, zero between calls
     if (impl == DM_IMPL_TCGEN05)
         st = fused_launch(c->fused, c->head, H, fa.B * fa.T, rows, map, mk, &n_slices, c->partials,
-                          logits_out, c->err, stream, &launches, &fa, c->err + 1,
-                          c->partials + (size_t)kMaxSlices * c->max_rows, &folded, nullptr, c->wait_limit, c->pdl, host);
+                          logits_out, c->err, stream, &launches, &fa, c->err + 1, best, &folded, nullptr,
+                          c->wait_limit, c->pdl, host, &best_reduced);
     else {
         if (host != nullptr) {
             st = launch_host_gather(host->h_src, host->h_bytes, host->draft_src, host->n_draft, host->h_dst,
@@ -172,9 +173,13 @@ int run_verify(dm_ctx* c, const void* H, int rows, const RowMap& map, const Mask
     }
     if (st != DM_OK) return st;
     if (!folded) {   // calls of several launches, and the CUDA-core family, finish in a kernel of their own
-        st = launch_finalize(c->partials, n_slices, rows, fa, stream);
+        st = best_reduced ? launch_finalize(best, 1, rows, fa, stream) : launch_finalize(c->partials, n_slices, rows, fa, stream);
         if (st != DM_OK) return st;
         ++launches;
+        if (best_reduced && cudaMemsetAsync(best, 0, (size_t)rows * sizeof(unsigned long long), stream) != cudaSuccess) {
+            cudaGetLastError();
+            return DM_ECUDA;
+        }
     }
     c->done_armed = host != nullptr && (folded || fa.B == 1);   // one block finishes the call and writes the word
     c->last_impl = impl;

@@ -1064,8 +1064,10 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
                  const RowMap& map, const MaskKey& mk, int* n_slices_out, unsigned long long* partials,
                  float* dbg_logits, uint32_t* err, cudaStream_t stream, int* launches_out,
                  const FinalizeArgs* fin, unsigned int* ticket, unsigned long long* best, bool* folded_out,
-                 unsigned long long* packed_out, long long wait_limit, bool allow_pdl, const HostInputs* host) {
+                 unsigned long long* packed_out, long long wait_limit, bool allow_pdl, const HostInputs* host,
+                 bool* best_reduced_out) {
     if (folded_out) *folded_out = false;
+    if (best_reduced_out) *best_reduced_out = false;
     if (fs == nullptr || !fused_supported(head, rows) || fs->geo[0].n_ctas + 1 > kMaxSlices) return DM_EUNSUPPORTED;
     // Slices of one-block launches: an even count (pairs need one); a CTA whose slice lies past the
     // end of W contributes empty partials.
@@ -1153,12 +1155,17 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         P.ticket = ticket;
         P.best = best;
         if (P.fold) { P.fin = *fin; if (folded_out) *folded_out = true; }
-        if (packed_out != nullptr && rows <= kMaxNPad) {
-            // one launch covers the call and the caller wants one packed word per path: reduce
-            // straight into the caller's array (which the caller has zeroed on this stream)
+        if (packed_out != nullptr) {
+            // the caller wants one packed word per path: reduce straight into the caller's array
+            // (which the caller has zeroed on this stream); every launch of the call has rows of its own
             P.fold = 2;
             P.best = packed_out;
             if (folded_out) *folded_out = true;
+        } else if (!P.fold && best != nullptr && best_reduced_out != nullptr) {
+            // a call of several launches: each reduces its rows into the per-row array; one small
+            // finalize kernel then reads one word per path (the caller zeroes the array afterwards)
+            P.fold = 2;
+            *best_reduced_out = true;
         }
         // Programmatic stream serialization, except when the row selection of the debug call could
         // itself be the output of the kernel ahead (it is read in the prologue).

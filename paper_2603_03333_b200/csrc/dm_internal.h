@@ -94,7 +94,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int n_hidd
                  const FinalizeArgs* fin = nullptr, unsigned int* ticket = nullptr,
                  unsigned long long* best = nullptr, bool* folded_out = nullptr,
                  unsigned long long* packed_out = nullptr, long long wait_limit = 0, bool allow_pdl = true,
-                 const HostInputs* host = nullptr);
+                 const HostInputs* host = nullptr, bool* best_reduced_out = nullptr);
 
 // The staged masked operand of the tensor-core kernel (Eq. 1 and the numerator of Eq. 2), written to `out`.
 int fused_debug_operand(const HeadDesc& head, const void* H, int rows, const RowMap& map, const MaskKey& mk,
