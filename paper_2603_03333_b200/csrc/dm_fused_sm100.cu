@@ -1,8 +1,9 @@
 // Fused sm_100a kernel for bf16 heads: Eq. 1 masks (Philox), Eq. 2 masking, Eq. 3 on tcgen05
 // tensor cores with fp32 accumulators in TMEM, and the argmax of Sec. 3.2 in the epilogue.  W is
 // streamed from HBM once per launch and no logit is written (except on request: the debug call
-// and the JS criterion ask for them).  For calls of up to 32 paths the masked hidden rows
-// exist in shared memory only; for wider calls they are staged once through global memory.
+// the JS criterion and nucleus sampling ask for them).  On heads whose vocabulary slices are a
+// single tile the masked hidden rows exist in shared memory only; on larger heads they are staged
+// once per call through global memory.  W tiles are loaded with an L2 evict-first policy.
 //
 // Work split.  The vocabulary is cut into one contiguous slice per CTA (one CTA per SM) and
 // each slice into equal tiles of `tile_rows` <= 128 vocabulary rows.  The MMA is "swapped": a
@@ -14,9 +15,9 @@
 // blocks (64 elements = one 128-byte swizzled row) are the outer loop and the tiles the inner
 // one, all accumulators of the group being live at once, while W streams through a ring of
 // TMA stages exactly once.  The masked operand of a block is needed once per group:
-//   - one group (the whole slice fits TMEM): builder warps generate the masks with Philox in
+//   - one group (single-tile slices): builder warps generate the masks with Philox in
 //     registers and write the masked rows of each block into a shared-memory ring, once per call;
-//   - several groups ("staged"): mask_operand_kernel has written the masked rows to a staging
+//   - several groups ("staged"): the mask pass ahead in the stream has written the masked rows to a staging
 //     buffer in global memory once per call.  W tiles and operand blocks share one ring of
 //     "steps": a step is the group's W tiles of one hidden-size block with the operand block
 //     behind them, one barrier for "all of it has landed" and one for "the MMAs are done with
