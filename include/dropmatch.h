@@ -138,7 +138,7 @@ int dropmatch_verify_batched(dm_ctx* ctx, const void* H, const int32_t* draft, i
  * Softmax(l / temperature) (equal probabilities: increasing id) up to and including the one whose
  * cumulative probability reaches top_p, and the draw is restricted to it.  The cut needs all logits
  * of a path at once: the head kernel writes them to the buffer that dm_enable_js reserves (call it
- * first with room for B*T*K rows, else DM_EWORKSPACE), and a second kernel, one block per path,
+ * first with room for B*T*K rows, else DM_EWORKSPACE), and a second kernel, one thread-block cluster per path,
  * finds the boundary by mass (fixed-point sums: the result does not depend on the order of
  * additions) and draws the token.  Sharded heads (dm_set_vocab_offset) are not supported here: the
  * nucleus is taken over this context's head.

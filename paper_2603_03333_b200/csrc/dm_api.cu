@@ -435,7 +435,7 @@ int dropmatch_verify_batched_sampled(dm_ctx* c, const void* H, const int32_t* dr
         return run_verify(c, H, rows, map, mk, fa, s);
     }
     // Nucleus: the cut needs all logits of a path at once.  The head kernel writes them to the
-    // context's logits buffer (its own argmax is not used), one block per path finds the nucleus
+    // context's logits buffer (its own argmax is not used), one cluster of blocks per path finds the nucleus
     // and draws the token, the finalize kernel does the rest.
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return DM_ECUDA; }
     if (rows > c->max_rows) return DM_EWORKSPACE;

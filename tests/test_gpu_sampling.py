@@ -77,6 +77,8 @@ NUCLEUS_CASES = [
     (wl.Config("n_peaked", d=256, V=5000, dtype=wl.BF16, B=2, T=2, K=8, p=0.1), 0.05, 0.3),    # peaked: one or two tokens
     (wl.Config("n_staged", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1), 1.0, 0.8),   # staged head kernel, 192 paths
     (wl.Config("n_tiny", d=64, V=37, dtype=wl.BF16, B=1, T=2, K=4, p=0.3), 1.0, 0.6),
+    (wl.Config("n_cluster8", d=128, V=60000, dtype=wl.BF16, B=1, T=1, K=8, p=0.1), 1.5, 0.9),   # eight CTAs per path
+    (wl.Config("n_cluster2", d=64, V=9000, dtype=wl.BF16, B=1, T=8, K=8, p=0.1), 1.0, 0.7),     # 64 paths: two CTAs per path
 ]
 
 
