@@ -775,24 +775,34 @@ mask_operand_by_position_kernel(const __nv_bfloat16* __restrict__ H, __nv_bfloat
                                 RowMap map, uint32_t key0, uint32_t key1, uint32_t thr,
                                 const int32_t* __restrict__ draft_src, int32_t* __restrict__ draft_dst, int n_draft) {
     ptx::griddep_launch_dependents();
-    ptx::griddep_wait();   // (see mask_operand_kernel)
     __shared__ uint4 s_h[32];
     const int chunks = d >> 3, tiles = (chunks + 31) >> 5;
     const int q = (int)(blockIdx.x / tiles), c = (int)(blockIdx.x % tiles) * 32 + (threadIdx.x & 31);
     const int pl = threadIdx.x >> 5;
+    const int kp = map.K + map.plain_extra;
+    // The mask of the thread's first path depends on indices only: it is drawn before the wait,
+    // while the kernel ahead drains (and, for a host-buffer call, before H has crossed the link).
+    uint32_t mbits0 = 0;
+    if (c < chunks && pl < kp) {
+        RowKey k0;
+        row_key(map, q * kp + pl, k0);
+        mbits0 = keep4((uint32_t)(2 * c), k0, key0, key1, thr) | (keep4((uint32_t)(2 * c + 1), k0, key0, key1, thr) << 4);
+    }
+    ptx::griddep_wait();   // (see mask_operand_kernel)
     if (draft_src != nullptr && blockIdx.x == 0)
         for (int x = threadIdx.x; x < n_draft; x += 256) draft_dst[x] = draft_src[x];
     if (pl == 0 && c < chunks) s_h[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(H + (size_t)q * d + c * 8));
     __syncthreads();
     if (c >= chunks) return;
     const uint4 hv = s_h[threadIdx.x & 31];
-    const int kp = map.K + map.plain_extra;
     for (int i = pl; i < kp; i += 8) {
         const int r = q * kp + i;
-        RowKey k;
-        row_key(map, r, k);   // always valid in the regular order
-        const uint32_t mbits = keep4((uint32_t)(2 * c), k, key0, key1, thr) |
-                               (keep4((uint32_t)(2 * c + 1), k, key0, key1, thr) << 4);
+        uint32_t mbits = mbits0;
+        if (i != pl) {
+            RowKey k;
+            row_key(map, r, k);   // always valid in the regular order
+            mbits = keep4((uint32_t)(2 * c), k, key0, key1, thr) | (keep4((uint32_t)(2 * c + 1), k, key0, key1, thr) << 4);
+        }
         uint4 o;
         o.x = hv.x & mask_pair(mbits);
         o.y = hv.y & mask_pair(mbits >> 2);
