@@ -63,6 +63,13 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
     int32_t* flag = sm + TK;       // chain: ok[T]; tree: test[N] then ok/depth packed [N]
     const size_t row0 = (size_t)b * TK;
     const size_t out0 = (size_t)b * a.T * a.K;
+    // The first loads of the routine do not depend on one another: the per-row word and the draft
+    // token of this thread are requested together with the error word (one round trip, not three).
+    const bool one_slice = n_slices == 1;
+    unsigned long long first_word = 0ull;
+    int32_t first_draft = 0;
+    if (one_slice && tid < TK) first_word = __ldcg(partials + row0 + tid);
+    if (a.N == 0 && a.draft != nullptr && tid < Td) first_draft = a.draft[(size_t)b * Td + tid];
     // A kernel of this call gave up on a wait (device error word set): the partial maxima are
     // incomplete.  Nothing may then look accepted to a consumer further down the stream: no token
     // (-1), empty histogram, accepted length 0 (the left-to-right rule rejects everything).
@@ -100,9 +107,13 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
     if (n_slices < 32) {
         for (int x = tid; x < TK; x += nthreads) {
             unsigned long long best = 0ull;
-            for (int s = 0; s < n_slices; ++s) {
-                unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x);
-                best = c > best ? c : best;
+            if (one_slice && x == tid) {
+                best = first_word;
+            } else {
+                for (int s = 0; s < n_slices; ++s) {
+                    unsigned long long c = __ldcg(partials + (size_t)s * rows + row0 + x);
+                    best = c > best ? c : best;
+                }
             }
             store_token(x, (int32_t)best_index(best));
         }
@@ -144,7 +155,7 @@ __device__ __forceinline__ void finalize_sequence(const unsigned long long* part
     if (a.N == 0) {
         for (int t = tid; t < Td; t += nthreads) {
             int hits;
-            bool ok = position_ok(toks + t * Kp, a.K, a.draft[(size_t)b * Td + t], a.rule, &hits);
+            bool ok = position_ok(toks + t * Kp, a.K, t == tid ? first_draft : a.draft[(size_t)b * Td + t], a.rule, &hits);
             flag[t] = ok;
             if (a.out_hits) a.out_hits[(size_t)b * Td + t] = hits;
         }
