@@ -536,7 +536,9 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // rounds a lane hands half of its packed (key, inverted index) columns to its partner
         // and keeps the maxima of the other half, so that 16 columns cost 16 exchanges, not 80.
         unsigned long long* my_best = s_best + ew * P.n_pad;
-        for (int n0 = 16 * set; n0 < P.n_pad; n0 += 16 * n_sets)
+        // accumulator columns past the launch's paths (padding of the MMA's N) are never read
+        const int n_cols = min(P.n_pad, (my_rows + 15) & ~15);
+        for (int n0 = 16 * set; n0 < n_cols; n0 += 16 * n_sets)
             if (lane < 16) my_best[n0 + lane] = 0ull;
         __syncwarp();
         const int m = lane_base + lane;
@@ -558,7 +560,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             const int slot0 = t0 % P.n_slots;
             const int v0 = v_cta0 + t0 * P.tile_rows + m;     // this lane's vocabulary row in tile t0
 #pragma unroll 1
-            for (int n0 = 16 * set; n0 < P.n_pad; n0 += 16 * n_sets) {
+            for (int n0 = 16 * set; n0 < n_cols; n0 += 16 * n_sets) {
                 float best[16];
                 int bv[16];
 #pragma unroll
