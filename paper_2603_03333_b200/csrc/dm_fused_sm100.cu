@@ -69,6 +69,9 @@ constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort 
 #ifndef DM_STAGED_MIN_NPAD
 #define DM_STAGED_MIN_NPAD 16   // slices of several tiles at least this wide are staged even if they would fit TMEM as one group
 #endif
+#ifndef DM_PAIR_GRAN
+#define DM_PAIR_GRAN 32        // operand rows of a pair launch are padded to a multiple of this (16 or 32)
+#endif
 #ifndef DM_PAIR_PAD_MIN
 #define DM_PAIR_PAD_MIN 64      // narrower pair launches are padded to this many accumulator columns
 #endif
@@ -832,7 +835,7 @@ struct FusedState {
     // builders, and one tensor map per box height n_pad = 16, 32, ..., 256 over it
     __nv_bfloat16* staging;
     int staging_rows;
-    CUtensorMap tmap_b[kMaxNPad / 16];
+    CUtensorMap tmap_b[kMaxNPad / 8];   // boxes of 8, 16, ..., 256 rows
 };
 
 namespace {
@@ -882,7 +885,7 @@ bool plan_smem(int rows, int tiles_per_cta, SmemPlan* out) {
     // on the Llama-3-8B head); the columns past the call's paths are computed and ignored.
     const bool force_staged = n_pad >= DM_STAGED_MIN_NPAD && tiles_per_cta > 1;
     best.pair = ((tiles_per_cta > kTmemCols / n_pad || force_staged) && n_pad >= kPairMinNPad) ? 1 : 0;
-    if (best.pair) n_pad = (rows + 31) & ~31;
+    if (best.pair) n_pad = (rows + DM_PAIR_GRAN - 1) & ~(DM_PAIR_GRAN - 1);
     if (best.pair && n_pad < DM_PAIR_PAD_MIN) n_pad = DM_PAIR_PAD_MIN;
     best.n_pad = n_pad;
     best.n_slots = kTmemCols / n_pad;
@@ -1009,10 +1012,10 @@ int fused_create(FusedState** out, const HeadDesc& head, int max_rows, int /*max
         if (cudaMalloc(&fs->staging, n) != cudaSuccess) { cudaGetLastError(); delete fs; return DM_ECUDA; }
         if (cudaMemset(fs->staging, 0, n) != cudaSuccess) { cudaGetLastError(); cudaFree(fs->staging); delete fs; return DM_ECUDA; }
         const cuuint64_t sdim[2] = {(cuuint64_t)head.d, (cuuint64_t)fs->staging_rows};
-        for (int n16 = 1; n16 <= kMaxNPad / 16; ++n16) {
-            const cuuint32_t sbox[2] = {(cuuint32_t)kBlockK, (cuuint32_t)(16 * n16)};
-            if (16 * n16 > fs->staging_rows) { fs->tmap_b[n16 - 1] = fs->tmap_b[0]; continue; }
-            r = encode(&fs->tmap_b[n16 - 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, fs->staging, sdim, gstride, sbox,
+        for (int n8 = 1; n8 <= kMaxNPad / 8; ++n8) {
+            const cuuint32_t sbox[2] = {(cuuint32_t)kBlockK, (cuuint32_t)(8 * n8)};
+            if (8 * n8 > fs->staging_rows) { fs->tmap_b[n8 - 1] = fs->tmap_b[0]; continue; }
+            r = encode(&fs->tmap_b[n8 - 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, fs->staging, sdim, gstride, sbox,
                        estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) { cudaFree(fs->staging); delete fs; return DM_ECUDA; }
@@ -1204,9 +1207,9 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         cfg.attrs = attrs;
         cfg.numAttrs = n_attrs;
         const cudaError_t launched =
-            plan.pair ? cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, geo.tmap_w, fs->tmap_b[P.n_pad / 32 - 1], P)
+            plan.pair ? cudaLaunchKernelEx(&cfg, fused_head_kernel<true>, geo.tmap_w, fs->tmap_b[P.n_pad / 16 - 1], P)
                       : cudaLaunchKernelEx(&cfg, fused_head_kernel<false>, geo.tmap_w,
-                                           plan.staged ? fs->tmap_b[P.n_pad / 16 - 1] : geo.tmap_w, P);
+                                           plan.staged ? fs->tmap_b[P.n_pad / 8 - 1] : geo.tmap_w, P);
         if (launched != cudaSuccess) {
             cudaGetLastError();
             return DM_ECUDA;
