@@ -31,8 +31,8 @@ WORKLOAD = "llama8b"   # Llama-3-8B-shaped head: the configuration the metric is
 
 # DRAM bytes (read + write) of one fused head-kernel launch on this workload, from the ncu capture
 # summarised in profiles/; None until a capture exists.
-NCU_TRAFFIC_BYTES = {"llama8b": 1051386000 + 3506000, "llama8b_k32": 1052965000 + 3706000,
-                     "llama8b_b2k32": 1078340000 + 5089000}
+NCU_TRAFFIC_BYTES = {"llama8b": 1051385000 + 1604000, "llama8b_k32": 1052995000 + 1725000,
+                     "llama8b_b2k32": 1080990000 + 2259000}
 
 
 def load_peaks():
