@@ -85,6 +85,8 @@ SMALL = [
     wl.Config("js_rows288", d=128, V=40000, dtype=wl.BF16, B=3, T=6, K=16, p=0.1),       # two head launches with logits
     wl.Config("js_k24", d=128, V=5000, dtype=wl.BF16, B=1, T=3, K=24, p=0.2),            # 17..32 paths in registers
     wl.Config("js_k40", d=128, V=2000, dtype=wl.BF16, B=1, T=2, K=40, p=0.2),            # more than fit: series by series
+    # many positions on a tiny vocabulary: the shares of the call do not fit the last block's scratch
+    wl.Config("js_many_pos", d=64, V=50, dtype=wl.BF16, B=2, T=50, K=2, p=0.2, draft_mode="toy"),
 ]
 
 
