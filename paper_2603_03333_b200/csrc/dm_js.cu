@@ -523,16 +523,18 @@ int launch_js_sweeps(const float* logits, const float* draft_prob, float* worksp
     if (cudaGetDevice(&dev) != cudaSuccess) return DM_ECUDA;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    static bool attr_set = false;
+    // the attribute belongs to the kernel on one device: remembered per device (the first 64)
+    static unsigned long long attr_set_on = 0ull;
+    const unsigned long long dev_bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
     const int smem_cap = 200 * 1024;
-    if (!attr_set) {
+    if ((attr_set_on & dev_bit) == 0ull) {
         if (cudaFuncSetAttribute(js_sweep_kernel<KMAX, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess ||
             cudaFuncSetAttribute(js_sweep_kernel<KMAX, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess ||
             cudaFuncSetAttribute(js_sweep_kernel<KMAX, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_cap) != cudaSuccess) {
             cudaGetLastError();
             return DM_ECUDA;
         }
-        attr_set = true;
+        attr_set_on |= dev_bit;
     }
     float2* part = reinterpret_cast<float2*>(workspace);
     JsAcceptArgs acc = acc_in;

@@ -323,13 +323,15 @@ int launch_nucleus_sample(const float* logits, int V, int rows, const RowMap& ma
     const size_t room = (size_t)smem_max - kNsFixedSmem - 1024;   // static arrays and slack
     const int stash_len = (size_t)chunk * sizeof(float) <= room ? chunk : (int)(room / sizeof(float));
     const size_t smem = kNsFixedSmem + (size_t)stash_len * sizeof(float);
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the attribute belongs to the kernel on one device: remembered per device (the first 64)
+    static unsigned long long attr_set_on = 0ull;
+    const unsigned long long dev_bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+    if ((attr_set_on & dev_bit) == 0ull) {
         if (cudaFuncSetAttribute(nucleus_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max - 1024) != cudaSuccess) {
             cudaGetLastError();
             return DM_ECUDA;
         }
-        attr_set = true;
+        attr_set_on |= dev_bit;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(rows * n_cta));
