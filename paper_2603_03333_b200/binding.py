@@ -94,19 +94,21 @@ def _check(status: int, where: str):
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    # the address as a plain int: ctypes converts it for pointer parameters, and building a
+    # c_void_p object per argument would cost more than the rest of the marshalling together
+    return None if t is None else t.data_ptr()
 
 
 _raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
 
 
-def _stream(device) -> ctypes.c_void_p:
+def _stream(device) -> int:
     # the handle of torch's current stream on `device` (the short way where this torch has it)
     if _raw_stream is not None:
         index = device if isinstance(device, int) else torch.device(device).index
         if index is not None:
-            return ctypes.c_void_p(_raw_stream(index))
-    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+            return _raw_stream(index)
+    return torch.cuda.current_stream(device).cuda_stream
 
 
 def _dev(t: torch.Tensor, dtype, what: str) -> torch.Tensor:
