@@ -69,6 +69,9 @@ constexpr int kBarBytes = 1024;             // mbarriers + TMEM address + abort 
 #ifndef DM_STAGED_MIN_NPAD
 #define DM_STAGED_MIN_NPAD 16   // slices of several tiles at least this wide are staged even if they would fit TMEM as one group
 #endif
+#ifndef DM_W_EVICT_FIRST_MIN_BYTES
+#define DM_W_EVICT_FIRST_MIN_BYTES 0   // heads larger than this many bytes stream W with the L2 evict-first policy
+#endif
 #ifndef DM_PAIR_GRAN
 #define DM_PAIR_GRAN 32        // operand rows of a pair launch are padded to a multiple of this (16 or 32)
 #endif
@@ -96,6 +99,7 @@ struct FusedParams {
     uint32_t step_bytes;
     int staged;       // masked operand comes from the staging buffer through TMA (tmap_b)
     int pdl;          // launched with programmatic stream serialization: see the griddep_wait() calls
+    int w_evict_first;   // W tiles are loaded with the L2 evict-first policy (heads larger than L2)
     long long wait_limit;   // clock cycles after which a wait on an mbarrier gives up (see dm_debug_set_wait_limit)
     int row_blocks;   // 1, or 2: two blocks of 256 paths share one pass over W (see fused_launch)
     RowMap map;
@@ -234,7 +238,7 @@ fused_head_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         // W is read once per launch: its lines go first when L2 needs room, so that the staged
         // operand, and the logits a call may write, stay there.  Not when two row blocks share the
         // stream: the second reader of a tile is meant to find it in L2.
-        const uint64_t w_policy = P.row_blocks == 1 ? ptx::l2_policy_evict_first() : ptx::l2_policy_evict_normal();
+        const uint64_t w_policy = (P.row_blocks == 1 && P.w_evict_first) ? ptx::l2_policy_evict_first() : ptx::l2_policy_evict_normal();
         if (P.staged) {
             // one step per (group, hidden-size block): the group's W tiles side by side
             for (int g = 0; g < n_groups; ++g) {
@@ -1186,6 +1190,7 @@ int fused_launch(FusedState* fs, const HeadDesc& head, const void* H, int /*n_hi
         // Programmatic stream serialization, except when the row selection of the debug call could
         // itself be the output of the kernel ahead (it is read in the prologue).
         P.pdl = (map.sel == nullptr && allow_pdl) ? 1 : 0;
+        P.w_evict_first = (size_t)head.V * head.d * sizeof(__nv_bfloat16) > (size_t)DM_W_EVICT_FIRST_MIN_BYTES ? 1 : 0;
         P.wait_limit = wait_limit > 0 ? wait_limit : kWaitLimitCycles;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)grid);
