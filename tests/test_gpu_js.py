@@ -140,3 +140,35 @@ def test_js_llama8b_full_size():
         assert not (tok_diff & (plain["gap"] >= NEAR_TIE)).any()
         pytest.skip("a near-tie flipped a token; divergences are checked by the other tests")
     _check(got, ref, draft, cfg)
+
+
+@pytest.mark.parametrize("cfg", [
+    wl.Config("js_graph_one", d=256, V=9000, dtype=wl.BF16, B=1, T=4, K=8, p=0.2),        # sweeps in one cooperative launch
+    wl.Config("js_graph_two", d=128, V=60000, dtype=wl.BF16, B=2, T=6, K=16, p=0.1),      # sweeps in two launches
+], ids=lambda c: c.name)
+def test_js_call_in_a_cuda_graph(cfg):
+    """dropmatch_verify_js only enqueues work: captured into a CUDA graph and replayed it gives the
+    eager call's results (the oracle referees the eager call in the tests above)."""
+    work = wl.make_workload(cfg, device=DEV)
+    n_pos = cfg.B * cfg.T
+    dp = wl.make_draft_probs(work.W, work.H.reshape(n_pos, cfg.d), np.linspace(0.02, 1.2, n_pos)).view(cfg.B, cfg.T, cfg.V)
+    ctx = pk.Context(0)
+    try:
+        ctx.set_head(work.W, max_rows=max(cfg.rows, 16), max_hidden_rows=n_pos)
+        ctx.enable_js(cfg.rows, n_pos)
+        want = to_np(ctx.verify_js(work.H, work.draft, dp, cfg.K, cfg.p, SEED, seq_base=2))
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            out = ctx.verify_js(work.H, work.draft, dp, cfg.K, cfg.p, SEED, seq_base=2)
+        for _ in range(3):
+            for t in out.values():
+                t.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            got = to_np(out)
+            for key in want:
+                assert np.array_equal(got[key], want[key], equal_nan=want[key].dtype.kind == "f"), key
+        assert ctx.device_error() == 0
+    finally:
+        ctx.close()
